@@ -58,10 +58,9 @@ typedef enum {
 /* Compute paths of qlinear_w4a16 (what ql_select_path returns, what qlinear_w4a16_path takes). */
 typedef enum {
   QL_PATH_AUTO = 0,
-  QL_PATH_FMA = 1,   /* CUDA-core fp32 FMA, for very small M */
   QL_PATH_MMA = 2,   /* warp-level bf16 tensor-core MMA (mma.sync), registers-resident operands */
   QL_PATH_TC5 = 3    /* tcgen05 bf16 MMA, weights written to tensor memory, accumulators in TMEM */
-} ql_path;
+} ql_path;            /* (1 is not used: a CUDA-core path would need M FMAs per weight and was not built) */
 
 const char* ql_status_str(int status);
 
@@ -75,11 +74,12 @@ size_t ql_packed_bytes(int K, int N, int g);
  * word).  Returns 0 for unsupported arguments.  Needs no device. */
 size_t ql_workspace_bytes(int M_max, int N_max);
 
-/* Zeroes the control words of a workspace (asynchronously, on `stream`).  Call once after
- * allocating the workspace, and again after a call reported QL_ERR_DEVICE_TIMEOUT.  The kernels
- * leave the control words zeroed when they finish, so no further initialisation is needed
- * between calls.  One workspace serves one stream at a time: calls that may overlap on the GPU
- * need separate workspaces. */
+/* Zeroes a workspace (asynchronously, on `stream`): its control words, and the partial-tile slots,
+ * whose entries carry a tag that must not look valid by accident.  Call once after allocating the
+ * workspace, and again after a call reported QL_ERR_DEVICE_TIMEOUT.  The kernels leave the control
+ * words zeroed when they finish, so no further initialisation is needed between calls.  One
+ * workspace serves one stream at a time: calls that may overlap on the GPU need separate
+ * workspaces. */
 int ql_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
 /* Reads the workspace's status word into *host_out (QL_OK or QL_ERR_DEVICE_TIMEOUT).
@@ -124,7 +124,7 @@ int qpack_w4_g128(const uint32_t* wq, const uint16_t* scale, const uint8_t* zero
  *   workspace   >= ql_workspace_bytes(M, N) bytes, initialised by ql_workspace_init
  *
  * Weights enter the tensor core as the exact integers q - z; the per-group scale multiplies the
- * fp32 group sum.  The path (FMA / MMA / TC5) is chosen from (M, K, N, g); see ql_select_path.
+ * fp32 group sum.  The path (MMA / TC5) is chosen from (M, K, N, g); see ql_select_path.
  * Errors: QL_ERR_NULL, QL_ERR_SHAPE, QL_ERR_ALIGN, QL_ERR_WORKSPACE, QL_ERR_CUDA.
  */
 int qlinear_w4a16(const void* packed, const uint16_t* X, uint16_t* Y, int32_t* argmax_out,
@@ -155,10 +155,13 @@ int ql_select_path(int M, int K, int N, int g);
  * The packed weights of every LINEAR must be complete before the call and must not change while
  * it runs: a linear may start streaming its weights while the operation before it finishes.
  * Runs of operations with M <= 16 and one group size execute as ONE cooperative launch of a
- * persistent kernel (glue folded into the neighbouring linears, gate/up pairs fused, operations
- * that share no buffer overlapped); its thread blocks wait for one another with bounded waits, so
- * a stream that is starved of SMs for more than 2 s reports QL_ERR_DEVICE_TIMEOUT in the status
- * word instead of hanging.  ql_stack_plan tells what a list turns into.  The call stages the fused
+ * persistent kernel.  A run of plain linears no two of which share a buffer (other than inputs
+ * both only read) and whose K is at most 24 groups is treated as one long stream of chunks cut
+ * into one contiguous piece per thread block; any other run is a chain - glue folded into the
+ * neighbouring linears, gate/up pairs fused, every operation waiting for the one before it.  The
+ * thread blocks wait for one another with bounded waits, so a stream that is starved of SMs for
+ * more than 2 s reports QL_ERR_DEVICE_TIMEOUT in the status word instead of hanging.
+ * ql_stack_plan tells what a list turns into.  The call stages the fused
  * operation descriptors from host memory into the workspace with an asynchronous copy, so it is
  * not meant to be recorded by stream capture.
  * Errors: as qlinear_w4a16, reported for the first offending operation; nothing is launched
@@ -192,7 +195,7 @@ int qlinear_stack_w4a16(const ql_op* ops, int n_ops,
  * them, [2] of which gate/up pairs run as one dual operation, [3] glue operations folded into their
  * neighbouring linears, [4] fused operations that do not wait for their predecessor, [5] linears
  * launched on their own, [6] glue operations launched on their own, [7] of the launches in [0],
- * those whose operations are pairwise independent plain linears and take the batch kernel.
+ * those whose operations are pairwise independent plain linears and run as one stream of chunks.
  */
 int ql_stack_plan(const ql_op* ops, int n_ops, void* workspace, size_t workspace_bytes, int counts[8]);
 
@@ -241,6 +244,15 @@ int ql_static_status(int* host_out, void* stream);
  * [ql_plan_first_chunk(.., i), ql_plan_first_chunk(.., i+1)); ql_plan_chunk_owner is the inverse. */
 uint32_t ql_plan_first_chunk(uint32_t total_chunks, uint32_t ncta, uint32_t cta);
 uint32_t ql_plan_chunk_owner(uint32_t total_chunks, uint32_t ncta, uint32_t chunk);
+
+/* Test hooks for the bounded waits of the persistent kernel (process-wide; not for production use).
+ * ql_debug_set_wait_budget_ns: budget of every wait inside qlinear_stack_w4a16 launches that
+ * follow (0 restores the default of 2 s).  ql_debug_no_release(i): in the launches that follow, the
+ * i-th fused operation of a launch does not publish its finished tiles, so the operation after it
+ * waits until its budget runs out, the status word becomes QL_ERR_DEVICE_TIMEOUT and the kernel
+ * runs to its end without hanging; -1 switches the hook off.  Nothing traps or faults. */
+void ql_debug_set_wait_budget_ns(uint64_t ns);
+void ql_debug_no_release(int fused_op);
 
 /* Number of kernels the library has launched since it was loaded (all entry points, this
  * process).  For benchmarks that report their launch count. */

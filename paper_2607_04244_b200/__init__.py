@@ -15,8 +15,8 @@ LIB_PATH = os.path.join(_PKG_DIR, "libqlinear_w4a16.so")
 QL_OK = 0
 QL_ERR_NULL, QL_ERR_SHAPE, QL_ERR_ALIGN, QL_ERR_UNSUPPORTED = 1, 2, 3, 4
 QL_ERR_WORKSPACE, QL_ERR_CUDA, QL_ERR_DEVICE_TIMEOUT = 5, 6, 7
-QL_PATH_AUTO, QL_PATH_FMA, QL_PATH_MMA, QL_PATH_TC5 = 0, 1, 2, 3
-PATH_NAMES = {QL_PATH_FMA: "fma", QL_PATH_MMA: "mma", QL_PATH_TC5: "tcgen05"}
+QL_PATH_AUTO, QL_PATH_MMA, QL_PATH_TC5 = 0, 2, 3
+PATH_NAMES = {QL_PATH_MMA: "mma", QL_PATH_TC5: "tcgen05"}
 QL_OP_LINEAR, QL_OP_UNIT_RMS, QL_OP_SILU_MUL_UNIT_RMS = 0, 1, 2
 
 EXPORTS = [
@@ -24,6 +24,7 @@ EXPORTS = [
     "ql_device_status_raw",
     "qpack_w4_g128", "qlinear_w4a16", "qlinear_w4a16_path", "ql_select_path", "qlinear_stack_w4a16",
     "qlinear_stack_w4a16_host", "ql_launch_count", "qlinear_w4a16_static", "ql_static_status", "ql_stack_plan", "ql_plan_first_chunk", "ql_plan_chunk_owner",
+    "ql_debug_set_wait_budget_ns", "ql_debug_no_release",
 ]
 
 
@@ -90,6 +91,10 @@ def load(path: str | None = None):
     for fn in (lib.ql_plan_first_chunk, lib.ql_plan_chunk_owner):
         fn.restype = ctypes.c_uint32
         fn.argtypes = [ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32]
+    lib.ql_debug_set_wait_budget_ns.restype = None
+    lib.ql_debug_set_wait_budget_ns.argtypes = [ctypes.c_uint64]
+    lib.ql_debug_no_release.restype = None
+    lib.ql_debug_no_release.argtypes = [i32]
     lib.ql_launch_count.restype = ctypes.c_uint64
     lib.ql_launch_count.argtypes = []
     _lib = lib
@@ -127,6 +132,14 @@ def ql_select_path(M: int, K: int, N: int, g: int) -> int:
 
 def ql_launch_count() -> int:
     return int(load().ql_launch_count())
+
+
+def ql_debug_set_wait_budget_ns(ns: int) -> None:
+    load().ql_debug_set_wait_budget_ns(ns)
+
+
+def ql_debug_no_release(fused_op: int) -> None:
+    load().ql_debug_no_release(fused_op)
 
 
 # ---- device entry points ----------------------------------------------------------------------

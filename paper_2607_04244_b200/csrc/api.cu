@@ -12,15 +12,16 @@ cudaError_t launch_qpack(const uint32_t*, const uint16_t*, const uint8_t*, int, 
 cudaError_t launch_linear_mma(LinearParams, cudaStream_t);
 cudaError_t launch_linear_tc5(LinearParams, int sms, cudaStream_t, bool pdl);
 bool tc5_supported(const LinearParams&, int sms);
-struct StackPlan { int ncta, n_x, n_stages, x_double; size_t smem; bool ok; };
+struct StackPlan { int ncta, n_x, n_stages; size_t smem; bool ok; };
+int stack_ncta(int sms);
 StackPlan stack_plan(const MegaOp* ops, int n_ops, int g, int sms);
 cudaError_t launch_stack_tc5(const StackParams& sp, int g, size_t smem, cudaStream_t stream);
-struct BatchPlan { int ncta, n_x, n_stages; size_t smem; bool ok; };
-BatchPlan batch_plan(const MegaOp* ops, int n_ops, int g, int sms);
-cudaError_t launch_batch_tc5(const StackParams& sp, int g, size_t smem, cudaStream_t stream);
 cudaError_t launch_unit_rms(const uint16_t*, const uint16_t*, uint16_t*, int, int, int, int, bool, cudaStream_t);
 
 static std::atomic<uint64_t> g_launches{0};
+static std::atomic<uint32_t> g_epoch{0};                  // stack-kernel launches: tags of split-K partial tiles
+static std::atomic<uint64_t> g_wait_ns{kWaitBudgetNs};    // budget of the stack kernel's bounded waits
+static std::atomic<int> g_no_release_op{-1};              // test hook: fused operation that does not publish its tiles
 
 static bool shape_ok(int M, int K, int N, int g) {
   if (M < 1 || M > 64) return false;
@@ -150,7 +151,10 @@ static MegaOp make_mega(const ql_op& o, const ql_op* second) {
   m.K = o.K; m.N = o.N; m.ld_in = o.ld_in; m.ld_out = o.ld_out; m.ld_xout = 0;
   m.n_tiles = o.N / kTileN; m.n_groups = o.K / o.g;
   m.total_chunks = (uint32_t)m.n_tiles * (uint32_t)m.n_groups;
+  m.flags = second ? kOpDual : 0;
   m.prologue = 0; m.src_tiles = 0; m.emit_ssq = 0;
+  m.cat_base = 0;
+  run_split(m.total_chunks, 1, m.nc, m.cq, m.cr);
   return m;
 }
 
@@ -180,12 +184,17 @@ static bool independent_ops(const MegaOp& prev, const MegaOp& cur, int M) {
   return true;
 }
 
+constexpr int kBatchMaxGroups = 24;   // K <= 24 groups: X of one operation (24 x 4.25 KB) beside a useful ring
+
 // True if the run is a list of plain linears no two of which share a buffer other than inputs
 // that both only read: such a run goes to the batch kernel, which overlaps its operations freely.
 static bool batchable(const std::vector<MegaOp>& mega, int M) {
   if (mega.size() < 2) return false;
   for (const MegaOp& m : mega)
     if (m.packed1 != nullptr || m.prologue != 0 || m.emit_ssq != 0 || m.argmax_out != nullptr || m.out0 == nullptr) return false;
+  // one CTA works through a long piece of the run: the X of a whole operation has to fit in shared memory
+  for (const MegaOp& m : mega)
+    if (m.n_groups > kBatchMaxGroups) return false;
   for (size_t a = 0; a < mega.size(); ++a)
     for (size_t b = a + 1; b < mega.size(); ++b)
       if (!independent_ops(mega[a], mega[b], M) || !independent_ops(mega[b], mega[a], M)) return false;
@@ -202,7 +211,7 @@ static bool is_dual(const ql_op* ops, int i, int n_ops) {
   return true;
 }
 
-// Operations per stack-kernel launch: their descriptors are kept in shared memory (128 B each).
+// Operations per stack-kernel launch (the partial-tile tags keep 9 bits for the operation number).
 constexpr int kStackRunOps = 256;
 
 // What the planner made of an operation list (ql_stack_plan reports it without launching).
@@ -233,32 +242,48 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
 
   auto flush = [&]() -> int {
     if (!mega.empty()) {
+      const int ncta = stack_ncta(sms);
+      // Independent plain linears form ONE run: their chunks are laid end to end and every CTA
+      // takes one contiguous piece.  Anything else is a chain: every operation is its own run and
+      // waits for the one before it.
+      const bool batch = batchable(mega, run_M);
+      if (batch) {
+        uint32_t total = 0;
+        for (MegaOp& m : mega) { m.cat_base = total; total += m.total_chunks; }
+        for (MegaOp& m : mega) run_split(total, (uint32_t)ncta, m.nc, m.cq, m.cr);
+      } else {
+        for (size_t j = 0; j < mega.size(); ++j) {
+          MegaOp& m = mega[j];
+          m.cat_base = 0;
+          run_split(m.total_chunks, (uint32_t)ncta, m.nc, m.cq, m.cr);
+          if (j > 0) m.flags |= kOpWait;
+        }
+      }
+      const int hook = g_no_release_op.load(std::memory_order_relaxed);
+      if (hook >= 0 && hook < (int)mega.size()) mega[hook].flags |= kOpNoRelease;
       StackPlan plan = stack_plan(mega.data(), (int)mega.size(), run_g, sms);
       if (!plan.ok) return QL_ERR_UNSUPPORTED;   // cannot happen: every operation was checked when it was added
-      BatchPlan bplan = {};
-      if (batchable(mega, run_M)) bplan = batch_plan(mega.data(), (int)mega.size(), run_g, sms);
-      if (bplan.ok) { plan.ncta = bplan.ncta; plan.n_x = bplan.n_x; plan.n_stages = bplan.n_stages; plan.smem = bplan.smem; plan.x_double = 1; }
       int n_tiles_cap = 1;
       for (const MegaOp& m : mega) n_tiles_cap = m.n_tiles > n_tiles_cap ? m.n_tiles : n_tiles_cap;
       StackParams sp = {};
       sp.ws = ws_carve(workspace, n_tiles_cap, 16);
       sp.ops = reinterpret_cast<const MegaOp*>(sp.ws.desc);
       sp.n_ops = (int)mega.size(); sp.M = run_M; sp.ncta = plan.ncta; sp.n_stages = plan.n_stages; sp.n_x = plan.n_x;
-      sp.x_double = plan.x_double;
+      sp.wait_ns = g_wait_ns.load(std::memory_order_relaxed);
       cnt.stack_launches += 1;
-      cnt.batch_launches += bplan.ok ? 1 : 0;
+      cnt.batch_launches += batch ? 1 : 0;
       cnt.fused_ops += (int)mega.size();
-      for (const MegaOp& m : mega) {
-        cnt.dual_ops += m.packed1 != nullptr;
+      for (size_t j = 0; j < mega.size(); ++j) {
+        const MegaOp& m = mega[j];
+        cnt.dual_ops += (m.flags & kOpDual) != 0;
         cnt.folded_glue += m.prologue != 0;
-        cnt.independent += (plan.x_double && m.indep) ? 1 : 0;
+        cnt.independent += (j > 0 && !(m.flags & kOpWait)) ? 1 : 0;
       }
-      for (MegaOp& m : mega) op_set_split(m, (uint32_t)plan.ncta);
       if (dry == nullptr) {
+        sp.epoch = g_epoch.fetch_add(1, std::memory_order_relaxed) + 1;
         if (cudaMemcpyAsync(sp.ws.desc, mega.data(), mega.size() * sizeof(MegaOp), cudaMemcpyHostToDevice, s) != cudaSuccess)
           return QL_ERR_CUDA;
-        if ((bplan.ok ? launch_batch_tc5(sp, run_g, plan.smem, s) : launch_stack_tc5(sp, run_g, plan.smem, s)) != cudaSuccess)
-          return QL_ERR_CUDA;
+        if (launch_stack_tc5(sp, run_g, plan.smem, s) != cudaSuccess) return QL_ERR_CUDA;
         g_launches.fetch_add(1, std::memory_order_relaxed);
       }
       mega.clear();
@@ -286,7 +311,11 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
         if (st != QL_OK) return st;
       }
       bool fits = o.M <= 16 && ws_total_bytes(m.n_tiles, 16) <= workspace_bytes;
-      if (fits) fits = stack_plan(&m, 1, o.g, sms).ok;
+      if (fits) {
+        MegaOp probe = m;                               // would it fit as a chained operation?
+        run_split(probe.total_chunks, (uint32_t)stack_ncta(sms), probe.nc, probe.cq, probe.cr);
+        fits = stack_plan(&probe, 1, o.g, sms).ok;
+      }
       if (fits && !mega.empty() && (o.M != run_M || o.g != run_g)) {
         const int st = flush();
         if (st != QL_OK) return st;
@@ -303,8 +332,10 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
         continue;
       }
       if (pend != nullptr) {
+        // (a gate/up pair that consumes a silu-mul product is not folded: its tiles would overwrite the
+        // fp32 product in the workspace while other CTAs still build their X from it)
         const bool fuse = !mega.empty() && pend->out == o.in0 && o.ld_in == pend->ld_out && o.K == pend->N && o.M == run_M &&
-                          o.g == run_g;
+                          o.g == run_g && !(dual && pend->kind == QL_OP_SILU_MUL_UNIT_RMS);
         if (fuse) {
           const int kind = pend->kind == QL_OP_SILU_MUL_UNIT_RMS ? 2 : 1;
           m.prologue = kind;
@@ -319,7 +350,6 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
         }
       }
       if (mega.empty()) { run_M = o.M; run_g = o.g; }
-      m.indep = (!mega.empty() && independent_ops(mega.back(), m, o.M)) ? 1 : 0;
       mega.push_back(m);
       if (dual) ++i;                                  // the second linear of the pair is part of this operation
     } else {
@@ -331,10 +361,10 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
       if (attach) {
         const MegaOp& prod = mega.back();
         if (o.kind == QL_OP_UNIT_RMS)
-          attach = prod.packed1 == nullptr && prod.out0 != nullptr && o.in0 == prod.out0 && o.ld_in == prod.ld_out &&
+          attach = !(prod.flags & kOpDual) && prod.out0 != nullptr && o.in0 == prod.out0 && o.ld_in == prod.ld_out &&
                    o.N % kTileN == 0 && o.N <= prod.N;
         else
-          attach = prod.packed1 != nullptr && o.in0 == prod.out0 && o.in1 == prod.out1 && o.N == prod.N && o.ld_in == prod.ld_out;
+          attach = (prod.flags & kOpDual) && o.in0 == prod.out0 && o.in1 == prod.out1 && o.N == prod.N && o.ld_in == prod.ld_out;
       }
       if (attach) {
         pend = &o;
@@ -388,7 +418,8 @@ int ql_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
   if (workspace == nullptr) return QL_ERR_NULL;
   if (workspace_bytes < kWsControlBytes) return QL_ERR_WORKSPACE;
   if (!aligned16(workspace)) return QL_ERR_ALIGN;
-  if (cudaMemsetAsync(workspace, 0, kWsControlBytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) return QL_ERR_CUDA;
+  // everything, not only the control words: the partial-tile slots carry tags, and a stale tag must never look valid
+  if (cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) return QL_ERR_CUDA;
   return QL_OK;
 }
 
@@ -441,7 +472,7 @@ int qlinear_w4a16_path(const void* packed, const uint16_t* X, uint16_t* Y, int32
   LinearParams p;
   int st = validate_linear(packed, X, K, Y, N, argmax_out, M, K, N, g, workspace, workspace_bytes);
   if (st != QL_OK) return st;
-  if (path < QL_PATH_AUTO || path > QL_PATH_TC5) return QL_ERR_UNSUPPORTED;
+  if (path != QL_PATH_AUTO && path != QL_PATH_MMA && path != QL_PATH_TC5) return QL_ERR_UNSUPPORTED;
   st = prepare_linear(p, packed, X, K, Y, N, argmax_out, M, K, N, g, workspace, workspace_bytes);
   if (st != QL_OK) return st;
   return run_linear(p, path, static_cast<cudaStream_t>(stream));
@@ -510,19 +541,20 @@ int ql_stack_plan(const ql_op* ops, int n_ops, void* workspace, size_t workspace
 
 uint32_t ql_plan_first_chunk(uint32_t total_chunks, uint32_t ncta, uint32_t cta) {
   if (total_chunks == 0 || ncta == 0) return 0;
-  MegaOp op = {};
-  op.total_chunks = total_chunks;
-  op_set_split(op, ncta);
-  return op_first_chunk(op, cta < op.nc ? cta : op.nc);
+  uint32_t nc, cq, cr;
+  run_split(total_chunks, ncta, nc, cq, cr);
+  return run_first_chunk(nc, cq, cr, cta < nc ? cta : nc);
 }
 
 uint32_t ql_plan_chunk_owner(uint32_t total_chunks, uint32_t ncta, uint32_t chunk) {
   if (total_chunks == 0 || ncta == 0 || chunk >= total_chunks) return 0;
-  MegaOp op = {};
-  op.total_chunks = total_chunks;
-  op_set_split(op, ncta);
-  return op_chunk_owner(op, chunk);
+  uint32_t nc, cq, cr;
+  run_split(total_chunks, ncta, nc, cq, cr);
+  return run_chunk_owner(nc, cq, cr, chunk);
 }
+
+void ql_debug_set_wait_budget_ns(uint64_t ns) { g_wait_ns.store(ns == 0 ? kWaitBudgetNs : ns, std::memory_order_relaxed); }
+void ql_debug_no_release(int fused_op) { g_no_release_op.store(fused_op, std::memory_order_relaxed); }
 
 uint64_t ql_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -27,7 +27,21 @@ struct LinearParams {
 
 // One fused operation of the stack kernel: a linear (or two linears that share their input, e.g.
 // gate and up), with the element-wise glue in front of it folded into how it loads X.
+//
+// Work split.  Operations are grouped into runs; the chunks of a run's operations, laid end to end,
+// are shared out in contiguous pieces among the first nc CTAs.  A run is either one operation
+// (chained operations: every CTA takes its share of every operation) or a list of independent
+// plain linears (each CTA then works through one long piece that touches one or two of them).
+// The first 32 bytes hold what every role reads at every operation.
+constexpr int kOpDual = 1;        // two matrices (packed0, packed1) share X
+constexpr int kOpWait = 2;        // X may be read only after operation j-1 has finished every tile
+constexpr int kOpNoRelease = 4;   // test hook: finished tiles are not published (the next operation's wait runs out)
 struct MegaOp {
+  uint32_t nc, cq, cr;     // CTA i owns run positions [i*cq + i*cr/nc, (i+1)*cq + (i+1)*cr/nc), i < nc
+  uint32_t cat_base;       // run position of this operation's chunk 0
+  uint32_t total_chunks;   // n_tiles * n_groups (per matrix)
+  int n_groups, n_tiles;
+  int flags;               // kOp* bits
   const uint8_t* packed0;  // packed weights
   const uint8_t* packed1;  // second matrix of a dual operation (same K, N, g), else nullptr
   const uint16_t* in0;     // X source, bf16 [M, ld_in]
@@ -36,19 +50,13 @@ struct MegaOp {
   uint16_t* out1;          // Y of matrix 1 (dual)
   uint16_t* xout;          // where the normalised X is written for the record (prologue != 0), else nullptr
   int32_t* argmax_out;     // [M] or nullptr
-  int K, N, ld_in, ld_out, ld_xout;
-  int n_tiles, n_groups;
-  uint32_t total_chunks;   // n_tiles * n_groups (per matrix)
+  int K, N, ld_in, ld_out;
+  int ld_xout;
   int prologue;            // 0: X = in0;  1: X = unit_rms(in0);  2: X = unit_rms(silu(in0) * in1)
   int src_tiles;           // column tiles of the producer that make up a normalised row (prologue != 0)
   int emit_ssq;            // 0: none; 1: per-tile row sums of bf16(Y)^2; 2: of (silu(bf16 Y0) * bf16 Y1)^2
-  int indep;               // 1: shares no buffer with the operation before it, so it need not wait for that one
-  // chunk split among the first nc CTAs without 64-bit division on the device:
-  // CTA i owns chunks [i*cq + i*cr/nc, (i+1)*cq + (i+1)*cr/nc),  cq = total/nc, cr = total%nc
-  uint32_t nc, cq, cr;
-  float nc_over_total;     // for a first guess of the CTA that owns a chunk
 };
-static_assert(sizeof(MegaOp) % 16 == 0 && sizeof(MegaOp) <= kOpDescBytes, "operation descriptor too large");
+static_assert(sizeof(MegaOp) == kOpDescBytes, "operation descriptor layout");
 
 struct StackParams {
   const MegaOp* ops;       // device copy of the descriptors (in the workspace)
@@ -56,27 +64,41 @@ struct StackParams {
   int M;
   int ncta;
   int n_stages;            // ring depth
-  int n_x;                 // X slots in shared memory (per buffer)
-  int x_double;            // 1: two X buffers, slot sets and counter ranges alternate between operations
+  int n_x;                 // X slots (groups) in shared memory
+  uint32_t epoch;          // launch number: partial tiles in the workspace carry (epoch, operation) tags
+  uint64_t wait_ns;        // budget of every bounded wait
   Workspace ws;
 };
 
-// Stack / batch kernels: first chunk of CTA i of an operation (32-bit arithmetic only; i*cr < 2^18).
-__host__ __device__ inline uint32_t op_first_chunk(const MegaOp& op, uint32_t i) { return i * op.cq + (i * op.cr) / op.nc; }
-// The CTA that owns chunk c: the largest i with op_first_chunk(i) <= c (float guess, exact correction).
-__host__ __device__ inline uint32_t op_chunk_owner(const MegaOp& op, uint32_t c) {
-  uint32_t i = (uint32_t)(((float)c + 0.5f) * op.nc_over_total);
-  if (i >= op.nc) i = op.nc - 1;
-  while (i > 0 && op_first_chunk(op, i) > c) --i;
-  while (i + 1 < op.nc && op_first_chunk(op, i + 1) <= c) ++i;
+// Run position of the first chunk of CTA i (32-bit arithmetic only; i*cr < 2^18).
+__host__ __device__ inline uint32_t run_first_chunk(uint32_t nc, uint32_t cq, uint32_t cr, uint32_t i) {
+  return i * cq + (i * cr) / nc;
+}
+// Chunks [lo, hi) of operation `op` (per matrix) that CTA i owns; lo == hi if none.
+__host__ __device__ inline void op_local_range(uint32_t nc, uint32_t cq, uint32_t cr, uint32_t cat_base, uint32_t total,
+                                               uint32_t i, uint32_t& lo, uint32_t& hi) {
+  lo = hi = 0;
+  if (i >= nc) return;
+  uint32_t a = run_first_chunk(nc, cq, cr, i), b = run_first_chunk(nc, cq, cr, i + 1);
+  const uint32_t top = cat_base + total;
+  if (a < cat_base) a = cat_base;
+  if (b > top) b = top;
+  if (a < b) { lo = a - cat_base; hi = b - cat_base; }
+}
+// The CTA that owns run position p: the largest i with run_first_chunk(i) <= p (float guess, exact correction).
+__host__ __device__ inline uint32_t run_chunk_owner(uint32_t nc, uint32_t cq, uint32_t cr, uint32_t p) {
+  const float total = (float)(nc * cq + cr);
+  uint32_t i = (uint32_t)(((float)p + 0.5f) * ((float)nc / total));
+  if (i >= nc) i = nc - 1;
+  while (i > 0 && run_first_chunk(nc, cq, cr, i) > p) --i;
+  while (i + 1 < nc && run_first_chunk(nc, cq, cr, i + 1) <= p) ++i;
   return i;
 }
-// Host: fill the split fields for a launch with ncta CTAs.
-inline void op_set_split(MegaOp& op, uint32_t ncta) {
-  op.nc = ncta < op.total_chunks ? ncta : op.total_chunks;
-  op.cq = op.total_chunks / op.nc;
-  op.cr = op.total_chunks % op.nc;
-  op.nc_over_total = (float)op.nc / (float)op.total_chunks;
+// Host: split a run of `run_total` chunks among ncta CTAs.
+inline void run_split(uint32_t run_total, uint32_t ncta, uint32_t& nc, uint32_t& cq, uint32_t& cr) {
+  nc = ncta < run_total ? ncta : run_total;
+  cq = run_total / nc;
+  cr = run_total % nc;
 }
 
 // First chunk of CTA i (64-bit product: total_chunks * ncta can exceed 2^32).

@@ -1,126 +1,202 @@
 // Persistent stack kernel: one cooperative launch runs a whole list of fused operations (the
-// projections of many decoder layers) with one CTA of 21 warps per SM, so that nothing of the hot
-// path crosses a kernel boundary:
-//   * the producer warp streams packed weights through the shared-memory ring without regard to
-//     operation boundaries - the weights of operation j+1 are already on chip while operation j
-//     still reduces its partial tiles;
-//   * operation j+1 reads its X only after operation j has finished every tile (a counter in the
-//     workspace, polled with a bounded wait);
+// projections of many decoder layers and the LM head) with one CTA of 22 warps per SM, so that
+// nothing of the hot path crosses a kernel boundary.
+//
+// Warps
+//   0-15   four unpack groups of 128 threads (thread n of a group = column n of a 128-column tile =
+//          tensor-memory lane n).  A group takes every fourth sub-chunk: it expands the int4 codes to
+//          the exact bf16 integers q - z, stores them into tensor memory as the A operand, later
+//          reads the 16 partial sums of its column back and adds them, scaled, to its accumulators.
+//          The same 512 threads build the X operand of an operation and finish its tiles.
+//   16     producer: one bulk copy (TMA engine, no tensor map, no multicast) per packed chunk into a
+//          ring of shared-memory stages; it runs ahead over operation boundaries, so the weights of
+//          operation j+1 are on chip while operation j is still being reduced.
+//   17-20  one MMA issuer per unpack group (a tcgen05.mma costs its issuing thread ~50-150 cycles).
+//   21     watcher: polls the counter of the previous operation, so that the other warps can work
+//          while they wait, and computes the row scales 1/rms from the per-tile sums of squares.
+//
+// What keeps a chain of dependent operations short (each one needs every output of the one before):
+//   * a group owns three half-chunk A buffers in tensor memory and unpacks the first one and a
+//     half chunks of operation j+1 BEFORE its X exists (the A operand depends on weights only);
+//     the issuers hold the MMAs back until X has been published;
+//   * waiting is done with relaxed loads (no fence per poll); the one acquire fence follows the
+//     successful poll;
+//   * split tiles: a contributor writes its partial sums as (value, tag) pairs and then sets a
+//     flag without a fence in between; the owner of the tile polls the flag, loads the pairs and
+//     checks every tag (a pair is one 8-byte store, so a matching tag proves the value), adding them
+//     in CTA order - deterministic, no floating-point atomics;
 //   * the glue between linears is folded in: a finished tile also leaves the row sums of squares
-//     of what the next operation normalises, and the next operation builds its X operand as
+//     of what the next operation normalises, and that operation builds its X operand as
 //     bf16(in * rsqrt(mean square)) (optionally of silu(gate) * up) while it loads it;
-//   * gate and up (two linears with one input) run as one dual operation: the even unpack groups
-//     take the gate chunks, the odd ones the up chunks of the same (tile, group) positions, they
-//     share the X operand, and the tile epilogue sees both results.
-// Warps: 0-15 four unpack groups of 128 threads (group w takes sub-chunks e = w mod 4), 16 the
-// producer, 17-20 one MMA issuer per unpack group.
-// The per-chunk pipeline (bulk copy -> unpack to tensor memory -> tcgen05.mma -> scale and
-// accumulate) is the one of the single-linear tcgen05 kernel.  M <= 16 only.
-#include <cstdio>
-#include <cstdlib>
-
+//   * gate and up (two linears with one input) run as one dual operation: even groups take the gate
+//     chunks, odd groups the up chunks of the same (tile, group) positions, they share X.
+// Every wait is bounded: on expiry the CTA records QL_ERR_DEVICE_TIMEOUT, raises its abort flag
+// (every later wait then falls through), lets its copies land, frees its tensor memory and exits.
+// M <= 16 only.
 #include "ql_params.h"
 
 namespace ql {
 
-constexpr int NWG = 4;                                 // unpack groups per CTA
-constexpr uint32_t kXWarps = (NWG - 1) * 4;            // warps that build the X operand (groups 1..3)
-constexpr int kStThreads = (NWG * 4 + 1 + NWG) * 32;   // 672
-constexpr int kStMaxStages = 32;
-constexpr uint32_t kStSmemBudget = 232448u;
+constexpr int NWG = 4;                                  // unpack groups per CTA
+constexpr int AH = 3;                                   // half-chunk A buffers per group
 constexpr int MP = 16;                                  // padded rows
-
-__host__ __device__ inline uint32_t st_fixed_smem() {
-  return (NWG - 1) * 512u * MP + 2u * kStMaxStages * 8u + 3u * NWG * 2u * 8u + 32u + 2048u + 2048u;
-}
+constexpr int kUnpackThreads = NWG * 128;               // 512
+constexpr int kWarpProducer = NWG * 4, kWarpIssuer0 = NWG * 4 + 1, kWarpWatcher = NWG * 4 + 1 + NWG;
+constexpr int kStThreads = (kWarpWatcher + 1) * 32;     // 704
+constexpr int kStMaxStages = 24;
+constexpr uint32_t kStSmemBudget = 232448u;
+constexpr uint32_t kXLbo = 16u * MP + 16u;              // bytes between K-adjacent 8x16-byte core matrices (+16: bank spread)
+__host__ __device__ constexpr uint32_t st_xslot_bytes(int g) { return (uint32_t)(g / 8) * kXLbo; }
+__host__ __device__ constexpr uint32_t st_fixed_smem() { return NWG * MP * 128u * 4u + 1024u; }
+constexpr uint32_t kSlotWords = 2u * MP * 128u;         // (value, tag) pairs of one CTA's partial tile, two matrices
 
 __device__ __forceinline__ float st_silu(float v) { return v / (1.f + __expf(-v)); }
-__device__ __forceinline__ float st_bf16_round(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 __device__ __forceinline__ void st_amax_merge(float& bv, int& bi, float v, int i) {
   if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
 }
-__device__ __forceinline__ int ld_acquire(const int* p) {
-  int v;
-  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-
-// Bounded wait until *ctr >= target (another CTA's progress).  On expiry: status word, abort flag.
 __device__ __forceinline__ int ld_relaxed(const int* p) {
   int v;
   asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ void wait_counter(const int* ctr, int target, volatile int* s_abort, int* status, int site) {
-  if (ld_acquire(ctr) >= target) return;
-  if (*s_abort) return;
+__device__ __forceinline__ void st_relaxed(int* p, int v) {
+  asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void red_relaxed_add(int* p, int v) {
+  asm volatile("red.relaxed.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void fence_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
+__device__ __forceinline__ void ld_pairs(const uint64_t* p, uint64_t& a, uint64_t& b) {
+  asm volatile("ld.relaxed.gpu.global.v2.b64 {%0,%1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
+}
+__device__ __forceinline__ void st_pairs(uint64_t* p, uint64_t a, uint64_t b) {
+  asm volatile("st.relaxed.gpu.global.v2.b64 [%0], {%1,%2};" ::"l"(p), "l"(a), "l"(b) : "memory");
+}
+__device__ __forceinline__ uint64_t tagged(float v, uint32_t tag) { return ((uint64_t)tag << 32) | (uint64_t)__float_as_uint(v); }
+
+struct WaitCtx {
+  volatile int* s_abort;
+  int* status;
+  uint64_t budget;
+};
+__device__ __forceinline__ void wait_fail(const WaitCtx& w, int site) {
+  *w.s_abort = 1;
+  atomicCAS(w.status, 0, kStatusTimeout | (site << 8) | ((int)blockIdx.x << 16));
+}
+// Bounded wait on an mbarrier phase (see mbar_wait; the budget is a launch parameter here).
+__device__ __forceinline__ void st_mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtx& w, int site) {
+  if (mbar_try_wait(bar, parity)) return;
+  if (*w.s_abort) return;
   const uint64_t t0 = globaltimer_ns();
   uint32_t spins = 0;
-  while (ld_acquire(ctr) < target) {
-    __nanosleep(64);
-    if ((++spins & 255u) == 0) {
-      if (*s_abort) return;
-      if (globaltimer_ns() - t0 > kWaitBudgetNs) {
-        *s_abort = 1;
-        atomicCAS(status, 0, kStatusTimeout | (site << 8) | ((int)blockIdx.x << 16));
-        return;
-      }
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 63u) == 0) {
+      if (*w.s_abort) return;
+      if (globaltimer_ns() - t0 > w.budget) { wait_fail(w, site); return; }
     }
   }
+}
+// Bounded wait until a global word written by another CTA satisfies `*p >= target` (geq) or `*p == target`.
+template <bool GEQ>
+__device__ __forceinline__ void wait_global(const int* p, int target, const WaitCtx& w, int site) {
+  int v = ld_relaxed(p);
+  if (GEQ ? v >= target : v == target) return;
+  if (*w.s_abort) return;
+  const uint64_t t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  for (;;) {
+    v = ld_relaxed(p);
+    if (GEQ ? v >= target : v == target) return;
+    if ((++spins & 15u) == 0) {
+      if (*w.s_abort) return;
+      if (globaltimer_ns() - t0 > w.budget) { wait_fail(w, site); return; }
+    }
+  }
+}
+// Bounded wait until a shared-memory word of this CTA exceeds `seen`.
+__device__ __forceinline__ void wait_shared_gt(volatile int* p, int seen, const WaitCtx& w, int site) {
+  if (*p > seen) return;
+  if (*w.s_abort) return;
+  const uint64_t t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  while (*p <= seen) {
+    if ((++spins & 63u) == 0) {
+      if (*w.s_abort) return;
+      if (globaltimer_ns() - t0 > w.budget) { wait_fail(w, site); return; }
+    }
+  }
+}
+
+// The fields of a descriptor that every role needs at every operation (two 16-byte loads through
+// the read-only path: the descriptors do not change while the kernel runs).
+struct OpHead {
+  uint32_t nc, cq, cr, cat_base, total_chunks;
+  int n_groups, n_tiles, flags;
+};
+__device__ __forceinline__ OpHead load_head(const MegaOp* op) {
+  const uint4 a = __ldg(reinterpret_cast<const uint4*>(op));
+  const uint4 b = __ldg(reinterpret_cast<const uint4*>(op) + 1);
+  OpHead h;
+  h.nc = a.x; h.cq = a.y; h.cr = a.z; h.cat_base = a.w;
+  h.total_chunks = b.x; h.n_groups = (int)b.y; h.n_tiles = (int)b.z; h.flags = (int)b.w;
+  return h;
+}
+template <typename T>
+__device__ __forceinline__ T* ldg_ptr(T* const* p) {
+  return reinterpret_cast<T*>(__ldg(reinterpret_cast<const unsigned long long*>(p)));
 }
 
 template <int G>
 __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_constant__ StackParams sp) {
   extern __shared__ __align__(1024) uint8_t smem[];
   constexpr uint32_t STAGE = align128(chunk_bytes(G));
-  constexpr uint32_t XSLOT = (uint32_t)MP * 2u * G;
-  constexpr int NK = G / 16;
-  constexpr int NC = G / 32;
+  constexpr uint32_t XSLOT = st_xslot_bytes(G);
+  constexpr int NK = G / 16;                            // MMAs per chunk
+  constexpr int NC = G / 32;                            // 16-byte code groups per column per chunk
+  constexpr uint32_t AHC = G / 4;                       // tensor-memory columns of one half-chunk A buffer
   constexpr uint32_t TMEM_COLS = 512;
-  constexpr uint32_t D_COL0 = NWG * (G / 2);           // first accumulator column
-  // tensor-memory columns: A buffer (group w, half h) at (2w+h)*(G/4); D buffer (group w, parity b) at D_COL0 + (2w+b)*MP
+  constexpr uint32_t D_COL0 = NWG * AH * AHC;           // first accumulator column
+  static_assert(D_COL0 + NWG * 2 * MP <= TMEM_COLS, "tensor memory layout");
+  // tensor-memory columns: A buffer (group w, slot s) at (w*AH + s)*AHC; D buffer (group w, parity b) at D_COL0 + (2w+b)*MP
   const int NS = sp.n_stages;
   uint8_t* ring = smem;
   uint8_t* xbuf = smem + (size_t)NS * STAGE;
-  const uint32_t XBUF = (uint32_t)sp.n_x * XSLOT;       // bytes of one X buffer
-  // the operation descriptors are read all the time (every phase of every warp): keep them on chip
-  const MegaOp* s_ops = reinterpret_cast<const MegaOp*>(xbuf + (size_t)(sp.x_double ? 2 : 1) * XBUF);
-  float* red = reinterpret_cast<float*>(xbuf + (size_t)(sp.x_double ? 2 : 1) * XBUF + (size_t)sp.n_ops * sizeof(MegaOp));  // [NWG-1][MP][128]
-  uint64_t* full = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(red) + (NWG - 1) * 512u * MP);
+  float* red = reinterpret_cast<float*>(xbuf + (size_t)sp.n_x * XSLOT);                 // [NWG][MP][128]
+  uint64_t* full = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(red) + NWG * MP * 128u * 4u);
   uint64_t* empty = full + kStMaxStages;
-  uint64_t* a_full = empty + kStMaxStages;             // [NWG][2]
-  uint64_t* a_empty = a_full + NWG * 2;                // [NWG][2]
-  uint64_t* d_full = a_empty + NWG * 2;                // [NWG][2]
-  float2* s_amax = reinterpret_cast<float2*>(d_full + NWG * 2 + 4);                             // [4][64]
-  int* s_flag = reinterpret_cast<int*>(s_amax + 4 * 64);                              // [0..15]
+  uint64_t* a_full = empty + kStMaxStages;              // [NWG][AH]
+  uint64_t* a_empty = a_full + NWG * AH;                // [NWG][AH]
+  uint64_t* d_full = a_empty + NWG * AH;                // [NWG][2]
+  uint64_t* x_full = d_full + NWG * 2;                  // [1]
+  float* s_inv = reinterpret_cast<float*>(x_full + 2);  // [16] 1/rms per row of the operation being prepared
+  int* s_flag = reinterpret_cast<int*>(s_inv + 16);     // [0..7]
   volatile int* s_abort = s_flag + 8;
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_flag + 9);
-  volatile uint32_t* s_xcount = reinterpret_cast<volatile uint32_t*>(s_flag + 10);
-  float* s_inv = reinterpret_cast<float*>(s_flag + 16);                               // [16] 1/rms per row
-  float* s_part = s_inv + 16;                                                         // [24][16] partial sums, then [4][16]
+  volatile int* s_dep = s_flag + 10;                    // operations whose predecessor is known to be complete
+  volatile int* s_invrdy = s_flag + 11;                 // operations whose 1/rms values are in s_inv
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const MegaOp* __restrict__ ops = sp.ops;
+  const WaitCtx wc = {s_abort, sp.ws.status, sp.wait_ns};
+  const uint32_t cta = blockIdx.x;
 
-  {
-    const uint4* src = reinterpret_cast<const uint4*>(sp.ops);
-    uint4* dst = reinterpret_cast<uint4*>(const_cast<MegaOp*>(s_ops));
-    for (int i = threadIdx.x; i < sp.n_ops * (int)(sizeof(MegaOp) / 16); i += kStThreads) dst[i] = src[i];
-  }
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], 4);
     }
-    for (int i = 0; i < NWG * 2; ++i) {
+    for (int i = 0; i < NWG * AH; ++i) {
       mbar_init(&a_full[i], 4);
       mbar_init(&a_empty[i], 1);
-      mbar_init(&d_full[i], 1);
     }
-    *s_xcount = 0;                                     // X operands published so far, times kXWarps (one count per X-duty warp)
+    for (int i = 0; i < NWG * 2; ++i) mbar_init(&d_full[i], 1);
+    mbar_init(x_full, NWG * 4);
     *s_abort = 0;
+    *s_dep = 0;
+    *s_invrdy = 0;
     fence_mbar_init();
   }
-  if (warp == NWG * 4 + 1) {
+  if (warp == kWarpIssuer0) {
     tmem_alloc(s_tmem, TMEM_COLS);
     tmem_relinquish();
   }
@@ -129,29 +205,33 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
   tc_fence_after_sync();
   const uint32_t tmem = *s_tmem;
 
-  if (warp == NWG * 4) {
+  if (warp == kWarpProducer) {
     // ------------------------------------------------------------------ producer: runs ahead over all operations
     if (lane == 0) {
       const uint64_t pol = policy_evict_first();
       const uint32_t cb = chunk_bytes(G);
       uint32_t s = 0, ph = 0, gs = 0;
       for (int j = 0; j < sp.n_ops; ++j) {
-        const MegaOp& op = s_ops[j];
-        const uint32_t nc = op.nc;                         // CTAs that share this operation (the first nc)
-        if (blockIdx.x >= nc) continue;
-        const uint32_t start = op_first_chunk(op, blockIdx.x);
-        const uint32_t end = op_first_chunk(op, blockIdx.x + 1);
-        const int nmat = op.packed1 != nullptr ? 2 : 1;
+        const OpHead h = load_head(ops + j);
+        uint32_t start, end;
+        op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
+        if (start >= end) continue;
+        const uint8_t* p0 = ldg_ptr(&ops[j].packed0);
+        const uint8_t* p1 = ldg_ptr(&ops[j].packed1);
+        const int nmat = (h.flags & kOpDual) ? 2 : 1;
         for (uint32_t c = start; c < end; ++c) {
           for (int mt = 0; mt < nmat; ++mt, ++gs) {
-            if (gs >= (uint32_t)NS) mbar_wait(&empty[s], ph ^ 1, s_abort, sp.ws.status, 1);
+            if (gs >= (uint32_t)NS) st_mbar_wait(&empty[s], ph ^ 1, wc, 1);
+            if (*s_abort) goto producer_done;            // never arm a stage that may still be in use
             mbar_arrive_expect_tx(&full[s], cb);
-            bulk_g2s_hint(ring + (size_t)s * STAGE, (mt ? op.packed1 : op.packed0) + (size_t)c * cb, cb, &full[s], pol);
+            bulk_g2s_hint(ring + (size_t)s * STAGE, (mt ? p1 : p0) + (size_t)c * cb, cb, &full[s], pol);
             if (++s == (uint32_t)NS) { s = 0; ph ^= 1; }
           }
         }
       }
+    producer_done:
       if (*s_abort) {
+        // a wait gave up somewhere: let this CTA's own copies land before it exits
         const uint32_t n = gs < (uint32_t)NS ? gs : (uint32_t)NS;
         for (uint32_t k = 0; k < n; ++k) {
           const uint32_t i2 = gs - 1 - k;
@@ -160,62 +240,92 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
         }
       }
     }
-  } else if (warp > NWG * 4) {
+  } else if (warp == kWarpWatcher) {
+    // ------------------------------------------------------------------ watcher: dependencies and row scales
+    for (int j = 0; j < sp.n_ops; ++j) {
+      const OpHead h = load_head(ops + j);
+      if (j > 0 && (h.flags & kOpWait)) {
+        if (lane == 0) {
+          const int need = __ldg(&ops[j - 1].n_tiles);
+          wait_global<true>(&sp.ws.op_done[j - 1], need, wc, 7);
+        }
+        __syncwarp();
+        fence_gpu();                                     // acquire: everything the finishers published
+      }
+      if (lane == 0) {
+        __threadfence_block();
+        *s_dep = j + 1;
+      }
+      const int prologue = __ldg(&ops[j].prologue);
+      uint32_t start, end;
+      op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
+      if (prologue != 0 && start < end) {
+        // 1/rms of every row from the per-tile sums of squares the producer operation left
+        // (fixed order: tiles of one parity ascending, then even + odd)
+        const int src_tiles = __ldg(&ops[j].src_tiles);
+        const float* ssq = sp.ws.ssq + (size_t)((j - 1) & 1) * sp.ws.n_tiles * 16;
+        const int row = lane & 15, half = lane >> 4;
+        float sum = 0.f;
+        for (int t0 = half; t0 < src_tiles; t0 += 16) {
+          float v[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) v[q] = (t0 + 2 * q < src_tiles) ? __ldcg(&ssq[(size_t)(t0 + 2 * q) * 16 + row]) : 0.f;
+#pragma unroll
+          for (int q = 0; q < 8; ++q) sum += v[q];
+        }
+        const float other = __shfl_xor_sync(0xffffffffu, sum, 16);
+        const float tot = half == 0 ? sum + other : other + sum;
+        if (lane < 16) s_inv[row] = rsqrtf(tot / (float)(src_tiles * kTileN));
+        __syncwarp();
+        if (lane == 0) {
+          __threadfence_block();
+          *s_invrdy = j + 1;
+        }
+      }
+      if (*s_abort) break;
+    }
+  } else if (warp >= kWarpIssuer0) {
     // ------------------------------------------------------------------ MMA issue for unpack group w
     if (lane == 0) {
       constexpr uint32_t idesc = tc_idesc_bf16_m128(MP);
-      const uint32_t w = warp - (NWG * 4 + 1);
-      const uint64_t desc0 = tc_smem_desc_kmajor(smem_u32(xbuf), MP * 16u, 128u);
-      constexpr uint32_t KSTEP = (2u * MP * 16u) >> 4;
+      const uint32_t w = warp - kWarpIssuer0;
+      const uint64_t desc0 = tc_smem_desc_kmajor(smem_u32(xbuf), kXLbo, 128u);
+      constexpr uint32_t KSTEP = (2u * kXLbo) >> 4;     // one MMA contracts 16 rows of K = two core matrices
       constexpr uint32_t SLOT = XSLOT >> 4;
-      const uint32_t a_base = tmem + 2 * w * (G / 4);
+      const uint32_t a_base = tmem + w * AH * AHC;
       uint32_t k = 0;                                  // chunks this group has handed over so far
-      uint32_t opc = 0;                                // operations this CTA took part in so far
+      uint32_t hs = 0;                                 // half-chunks
+      uint32_t xops = 0;                               // operations this CTA took part in so far
       for (int j = 0; j < sp.n_ops; ++j) {
-        const MegaOp& op = s_ops[j];
-        const uint32_t nc = op.nc;
-        if (blockIdx.x >= nc) continue;
-        const uint32_t start = op_first_chunk(op, blockIdx.x);
-        const uint32_t end = op_first_chunk(op, blockIdx.x + 1);
-        const bool dual = op.packed1 != nullptr;
-        const uint32_t Gn = op.n_groups;
-        // sub-chunk e of the operation: chunk start + (dual ? e >> 1 : e); this group takes e = w, w+NWG, ...
+        const OpHead h = load_head(ops + j);
+        uint32_t start, end;
+        op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
+        if (start >= end) continue;
+        const bool dual = (h.flags & kOpDual) != 0;
+        const uint32_t Gn = (uint32_t)h.n_groups;
         const uint32_t n_sub = (end - start) * (dual ? 2u : 1u);
-        // X of this operation is in shared memory once the 12 X-duty warps have each counted it in
-        ++opc;
-        if (w < n_sub) {
-          if (*s_xcount < kXWarps * opc && !*s_abort) {
-            const uint64_t t0 = globaltimer_ns();
-            uint32_t spins = 0;
-            while (*s_xcount < kXWarps * opc) {
-              if ((++spins & 255u) == 0) {
-                if (*s_abort) break;
-                if (globaltimer_ns() - t0 > kWaitBudgetNs) {
-                  *s_abort = 1;
-                  atomicCAS(sp.ws.status, 0, kStatusTimeout | (2 << 8) | ((int)blockIdx.x << 16));
-                  break;
-                }
-              }
-            }
-          }
-          __threadfence_block();
-          tc_fence_after_sync();
-        }
+        ++xops;
+        bool first = true;
         for (uint32_t e = w; e < n_sub; e += NWG, ++k) {
           uint32_t xk = dual ? (e >> 1) : e;           // X slot = chunk number within the CTA, modulo the group count
           xk = xk % Gn;
           const uint32_t d_tmem = tmem + D_COL0 + (2 * w + (k & 1)) * MP;
-          const uint64_t xdesc = desc0 + (uint64_t)(xk * SLOT + ((sp.x_double && (j & 1)) ? (XBUF >> 4) : 0u));
+          const uint64_t xdesc = desc0 + (uint64_t)(xk * SLOT);
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            mbar_wait(&a_full[2 * w + h], k & 1, s_abort, sp.ws.status, 3);
+          for (int hh = 0; hh < 2; ++hh, ++hs) {
+            const uint32_t slot = hs % AH;
+            st_mbar_wait(&a_full[w * AH + slot], (hs / AH) & 1, wc, 3);
+            if (first) {
+              st_mbar_wait(x_full, (xops - 1) & 1, wc, 2);   // X of this operation is in shared memory
+              first = false;
+            }
             tc_fence_after_sync();
 #pragma unroll
             for (int jj = 0; jj < NK / 2; ++jj) {
-              const int jk = h * (NK / 2) + jj;
-              tc_mma_ts_f16(d_tmem, a_base + h * (G / 4) + 8 * jj, xdesc + (uint64_t)(jk * KSTEP), idesc, jk > 0 ? 1u : 0u);
+              const int jk = hh * (NK / 2) + jj;
+              tc_mma_ts_f16(d_tmem, a_base + slot * AHC + 8 * jj, xdesc + (uint64_t)(jk * KSTEP), idesc, jk > 0 ? 1u : 0u);
             }
-            tc_commit(&a_empty[2 * w + h]);
+            tc_commit(&a_empty[w * AH + slot]);
           }
           tc_commit(&d_full[2 * w + (k & 1)]);
         }
@@ -226,18 +336,18 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
     const int w = warp >> 2;
     const int wq = warp & 3;
     const int n = wq * 32 + lane;                      // column inside the tile = TMEM lane
-    const int t384 = tid - 128;                        // index among groups 1..3 (X duty)
     const uint32_t tlane = tmem + ((uint32_t)(wq * 32) << 16);
-    const uint32_t a_addr = tlane + 2 * w * (G / 4);
+    const uint32_t a_addr = tlane + w * AH * AHC;
     const uint32_t d_addr = tlane + D_COL0 + 2 * w * MP;
-    const size_t slot_f = ws_slot_floats(MP);
+    uint64_t* my_slot = reinterpret_cast<uint64_t*>(sp.ws.slots) + (size_t)cta * kSlotWords;
     uint32_t stg = 0, sph = 0;                          // ring stage / phase of the next sub-chunk (any group's)
     uint32_t kloc = 0;                                  // chunks this group has handed to the tensor core
+    uint32_t hs = 0;                                    // half-chunks this group has stored
     float acc[MP];
 
     auto drain = [&](uint32_t kq, float s_q) {
       const uint32_t b = kq & 1;
-      mbar_wait(&d_full[2 * w + b], (kq >> 1) & 1, s_abort, sp.ws.status, 4);
+      st_mbar_wait(&d_full[2 * w + b], (kq >> 1) & 1, wc, 4);
       tc_fence_after_sync();
       float d[16];
       tmem_ld16(d_addr + b * MP, d);
@@ -247,97 +357,91 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
     };
 
     for (int j = 0; j < sp.n_ops; ++j) {
-      const MegaOp& op = s_ops[j];
-      const uint32_t nc = op.nc;                         // CTAs that share this operation (the first nc)
-      if (blockIdx.x >= nc) continue;
-      const uint32_t start = op_first_chunk(op, blockIdx.x);
-      const uint32_t end = op_first_chunk(op, blockIdx.x + 1);
-      const bool dual = op.packed1 != nullptr;
-      const uint32_t Gn = op.n_groups;
+      const OpHead h = load_head(ops + j);
+      uint32_t start, end;
+      op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
+      if (start >= end) continue;
+      const MegaOp* op = ops + j;
+      const bool dual = (h.flags & kOpDual) != 0;
+      const uint32_t Gn = (uint32_t)h.n_groups;
       const uint32_t my_chunks = end - start;
-      const int par = sp.x_double ? (j & 1) : 0;         // which X buffer, slot set and counter range
-      uint8_t* xb = xbuf + (size_t)par * XBUF;
-      float* slots = sp.ws.slots + (size_t)par * (kMaxCtas / 2) * 2 * slot_f;
-      int* tile_cnt = sp.ws.tile_cnt + par * (kMaxTiles / 2);   // used as one flag per (CTA, segment) partial slot
+      const uint32_t tag = (sp.epoch << 9) | (uint32_t)(j + 1);
+      bool x_done = false;
+      uint32_t pre = 0;                                 // half-chunks of this operation stored before its X exists
 
-      if (w != 0) {
-        // -------- X duty (groups 1..3, 384 threads): wait for the previous operation, build X --------
-        constexpr uint32_t UPS = (uint32_t)MP * (G / 8);   // 16-byte units per slot
+      // -------- X duty (all 512 threads): wait for the previous operation, build the X operand --------
+      auto x_duty = [&]() {
+        constexpr uint32_t UPG = (uint32_t)MP * (G / 8);   // 16-byte units per group
         const uint32_t n_x = min(my_chunks, Gn);
         const uint32_t g_first = start % Gn;
-        const uint32_t n_units = n_x * UPS;
-        if (op.prologue == 0) {
-          if (j > 0) {
-            // one thread of the CTA polls the counters; the other 383 wait at a barrier.  The operation
-            // two back must be complete before its X buffer, slots and counters are reused; the one
-            // just before only if this operation consumes or overwrites something of it.
-            if (t384 == 0) {
-              if (j > 1) wait_counter(&sp.ws.op_done[j - 2], s_ops[j - 2].n_tiles, s_abort, sp.ws.status, 8);
-              if (!(sp.x_double && op.indep)) wait_counter(&sp.ws.op_done[j - 1], s_ops[j - 1].n_tiles, s_abort, sp.ws.status, 7);
-            }
-            named_bar_sync(3, 384);
-          }
-          for (uint32_t idx = t384; idx < n_units; idx += 384) {
-            const uint32_t k = idx / UPS, u = idx % UPS;
-            const uint32_t ku = u / MP, m = u % MP;
+        const uint32_t n_units = n_x * UPG;
+        const int prologue = __ldg(&op->prologue);
+        const int ld_in = __ldg(&op->ld_in);
+        const uint16_t* in0 = ldg_ptr(&op->in0);
+        // unit idx: slot k = idx / UPG, row m = (idx / (G/8)) % MP, k-unit ku = idx % (G/8): lanes run along K
+        auto unit_addr = [&](uint32_t k, uint32_t m, uint32_t ku) -> uint8_t* {
+          return xbuf + (size_t)k * XSLOT + ku * kXLbo + (m >> 3) * 128u + (m & 7u) * 16u;
+        };
+        wait_shared_gt(s_dep, j, wc, 8);
+        __threadfence_block();
+        if (prologue == 0) {
+          for (uint32_t idx = tid; idx < n_units; idx += kUnpackThreads) {
+            const uint32_t k = idx / UPG, r = idx % UPG;
+            const uint32_t m = r / (G / 8), ku = r % (G / 8);
             uint32_t Gi = g_first + k;
             if (Gi >= Gn) Gi -= Gn;
             const bool live = (int)m < sp.M;
-            cp_async16(xb + (size_t)k * XSLOT + (size_t)u * 16,
-                       live ? (op.in0 + (size_t)m * op.ld_in + (size_t)Gi * G + ku * 8) : op.in0, live ? 16u : 0u);
+            cp_async16(unit_addr(k, m, ku), live ? (in0 + (size_t)m * ld_in + (size_t)Gi * G + ku * 8) : in0, live ? 16u : 0u);
           }
           asm volatile("cp.async.wait_all;" ::: "memory");
         } else {
           // X = bf16(v * 1/rms): v is the producer's bf16 output (prologue 1) or the fp32 product
           // silu(gate) * up it left in the workspace (prologue 2).  The loads of a batch are all
-          // issued before any is used, and the first batch is in flight while 1/rms is computed
-          // from the per-tile sums of squares (fixed summation order).
+          // issued before any is used; 1/rms arrives from the watcher meanwhile.
           constexpr int XB = 4;
+          const bool from_act = (prologue == 2);
           const float* act = sp.ws.act;
-          uint4 ra[XB], rb[XB];
-          uint32_t kk[XB], uu[XB], gg[XB];
-          const uint4* pa[XB];                             // source of each unit of the batch (nullptr: zero)
-          const bool from_act = (op.prologue == 2);
-          // addresses of a batch (everything that does not need the producer's data)
-          auto prep_batch = [&](uint32_t base) {
+          const int K = __ldg(&op->K);
+          uint16_t* xout = ldg_ptr(&op->xout);
+          const int ld_xout = __ldg(&op->ld_xout);
+          bool have_inv = false;
+          for (uint32_t base = tid; base < n_units; base += kUnpackThreads * XB) {
+            uint4 ra[XB], rb[XB];
+            uint32_t kk[XB], mm[XB], uu[XB], gg[XB];
 #pragma unroll
             for (int q = 0; q < XB; ++q) {
-              const uint32_t idx = base + q * 384;
+              const uint32_t idx = base + q * kUnpackThreads;
               const bool in_range = idx < n_units;
-              const uint32_t k = in_range ? idx / UPS : 0, u = idx % UPS;
+              const uint32_t k = in_range ? idx / UPG : 0, r = idx % UPG;
+              const uint32_t m = r / (G / 8), ku = r % (G / 8);
               uint32_t Gi = g_first + k;
               if (Gi >= Gn) Gi -= Gn;
-              kk[q] = k; uu[q] = u; gg[q] = Gi;
-              const uint32_t ku = u / MP, m = u % MP;
-              pa[q] = nullptr;
+              kk[q] = k; mm[q] = m; uu[q] = ku; gg[q] = Gi;
+              ra[q] = make_uint4(0u, 0u, 0u, 0u); rb[q] = ra[q];
               if (in_range && (int)m < sp.M) {
                 const size_t col0 = (size_t)Gi * G + ku * 8;
-                // the workspace copy of silu(gate)*up is dense [M][K]; the producer's bf16 output has its own leading dimension
-                pa[q] = from_act ? reinterpret_cast<const uint4*>(act + (size_t)m * op.K + col0)
-                                 : reinterpret_cast<const uint4*>(op.in0 + (size_t)m * op.ld_in + col0);
+                if (from_act) {
+                  const uint4* p = reinterpret_cast<const uint4*>(act + (size_t)m * K + col0);
+                  ra[q] = __ldcg(p);
+                  rb[q] = __ldcg(p + 1);
+                } else {
+                  ra[q] = __ldcg(reinterpret_cast<const uint4*>(in0 + (size_t)m * ld_in + col0));
+                }
               }
             }
-          };
-          auto issue_batch = [&]() {
-#pragma unroll
-            for (int q = 0; q < XB; ++q) {
-              ra[q] = make_uint4(0u, 0u, 0u, 0u); rb[q] = ra[q];
-              if (pa[q] != nullptr) {
-                ra[q] = __ldcg(pa[q]);
-                if (from_act) rb[q] = __ldcg(pa[q] + 1);
-              }
+            if (!have_inv) {
+              wait_shared_gt(s_invrdy, j, wc, 9);
+              __threadfence_block();
+              have_inv = true;
             }
-          };
-          auto store_batch = [&](uint32_t base) {
 #pragma unroll
             for (int q = 0; q < XB; ++q) {
-              const uint32_t idx = base + q * 384;
+              const uint32_t idx = base + q * kUnpackThreads;
               if (idx >= n_units) continue;
-              const uint32_t ku = uu[q] / MP, m = uu[q] % MP;
               uint4 o = make_uint4(0u, 0u, 0u, 0u);
-              if ((int)m < sp.M) {
-                const float inv = s_inv[m];
-                if (op.prologue == 1) {
+              if ((int)mm[q] < sp.M) {
+                const float inv = s_inv[mm[q]];
+                if (!from_act) {
                   o.x = pack_bf16x2_rn(bf16lo_to_f32(ra[q].x) * inv, bf16hi_to_f32(ra[q].x) * inv);
                   o.y = pack_bf16x2_rn(bf16lo_to_f32(ra[q].y) * inv, bf16hi_to_f32(ra[q].y) * inv);
                   o.z = pack_bf16x2_rn(bf16lo_to_f32(ra[q].z) * inv, bf16hi_to_f32(ra[q].z) * inv);
@@ -349,62 +453,21 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
                   o.w = pack_bf16x2_rn(__uint_as_float(rb[q].z) * inv, __uint_as_float(rb[q].w) * inv);
                 }
                 // the CTA that owns (tile 0, group Gi) writes the normalised X out for the record
-                if (op.xout != nullptr && start + kk[q] < Gn)
-                  *reinterpret_cast<uint4*>(op.xout + (size_t)m * op.ld_xout + (size_t)gg[q] * G + ku * 8) = o;
+                if (xout != nullptr && start + kk[q] < Gn)
+                  *reinterpret_cast<uint4*>(xout + (size_t)mm[q] * ld_xout + (size_t)gg[q] * G + uu[q] * 8) = o;
               }
-              *reinterpret_cast<uint4*>(xb + (size_t)kk[q] * XSLOT + (size_t)uu[q] * 16) = o;
+              *reinterpret_cast<uint4*>(unit_addr(kk[q], mm[q], uu[q])) = o;
             }
-          };
-          // sums of squares of this thread's share of the producer's tiles, and the first batch of X
-          const float* ssq = sp.ws.ssq + (size_t)((j - 1) & 1) * sp.ws.n_tiles * 16;
-          const int row = t384 & 15, part = t384 >> 4;     // 24 parts
-          prep_batch(t384);
-          if (j > 0) {
-            // one thread of the CTA polls the counters; the other 383 wait at a barrier.  The operation
-            // two back must be complete before its X buffer, slots and counters are reused; the one
-            // just before only if this operation consumes or overwrites something of it.
-            if (t384 == 0) {
-              if (j > 1) wait_counter(&sp.ws.op_done[j - 2], s_ops[j - 2].n_tiles, s_abort, sp.ws.status, 8);
-              if (!(sp.x_double && op.indep)) wait_counter(&sp.ws.op_done[j - 1], s_ops[j - 1].n_tiles, s_abort, sp.ws.status, 7);
-            }
-            named_bar_sync(3, 384);
-          }
-          float sv[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-          for (int q = 0; q < 4; ++q)
-            if (part + 24 * q < op.src_tiles) sv[q] = __ldcg(&ssq[(size_t)(part + 24 * q) * 16 + row]);
-          issue_batch();
-          float sacc = ((sv[0] + sv[1]) + sv[2]) + sv[3];
-          for (int tt = part + 96; tt < op.src_tiles; tt += 24) sacc += __ldcg(&ssq[(size_t)tt * 16 + row]);
-          s_part[part * 16 + row] = sacc;
-          named_bar_sync(3, 384);
-          if (t384 < 64) {
-            // 4 threads per row, 6 partial sums each, combined in a fixed order
-            const int r = t384 >> 2, c = t384 & 3;
-            float tot = 0.f;
-#pragma unroll
-            for (int q = 0; q < 6; ++q) tot += s_part[(c * 6 + q) * 16 + r];
-            tot += __shfl_xor_sync(0xffffffffu, tot, 1);
-            tot += __shfl_xor_sync(0xffffffffu, tot, 2);
-            if (c == 0) s_inv[r] = rsqrtf(tot / (float)(op.src_tiles * kTileN));
-          }
-          named_bar_sync(3, 384);
-          store_batch(t384);
-          for (uint32_t base = t384 + 384 * XB; base < n_units; base += 384 * XB) {
-            prep_batch(base);
-            issue_batch();
-            store_batch(base);
           }
         }
         fence_proxy_async();
-        __threadfence_block();
         __syncwarp();
-        if (lane == 0) atomicAdd(const_cast<uint32_t*>(s_xcount), 1u);
-      }
+        if (lane == 0) mbar_arrive(x_full);
+        x_done = true;
+      };
 
       // -------- chunks of this operation --------
       uint32_t pos = start, e = 0;                      // e: sub-chunk counter of the operation (this CTA)
-      int seg = 0;
       while (pos < end) {
         const uint32_t T = pos / Gn;
         const uint32_t g0 = pos - T * Gn;
@@ -421,31 +484,35 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
           if (++stg == (uint32_t)NS) { stg = 0; sph ^= 1; }
           if ((int)(e % NWG) != w) continue;
           const uint8_t* st = ring + (size_t)my_stage * STAGE;
-          mbar_wait(&full[my_stage], my_phase, s_abort, sp.ws.status, 5);
+          st_mbar_wait(&full[my_stage], my_phase, wc, 5);
           const float sc = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(st + 64 * G)[n] << 16);
           const uint32_t z = (reinterpret_cast<const uint32_t*>(st + 64 * G + 256)[n >> 3] >> (4 * (n & 7))) & 0xFu;
           const uint32_t zb = 0x43004300u | z | (z << 16);
           const uint4* wst = reinterpret_cast<const uint4*>(st);
           if (n_pend == 2) { drain(kloc - 2, s_p2); n_pend = 1; }
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            if (kloc > 0) {
-              mbar_wait(&a_empty[2 * w + h], (kloc - 1) & 1, s_abort, sp.ws.status, 6);
+          for (int hh = 0; hh < 2; ++hh, ++hs) {
+            // the A buffers hold AH half-chunks: whatever fits is unpacked before X exists, then
+            // the group turns to the X operand, whose MMAs free the buffers again
+            if (!x_done && pre == AH) x_duty();
+            ++pre;
+            const uint32_t slot = hs % AH;
+            if (hs >= AH) {
+              st_mbar_wait(&a_empty[w * AH + slot], ((hs / AH) - 1) & 1, wc, 6);
               tc_fence_after_sync();
             }
 #pragma unroll
             for (int cc = 0; cc < NC / 2; ++cc) {
               uint32_t v[16];
-
-              unpack_codes32(wst[(h * (NC / 2) + cc) * kTileN + n], zb, v);
-              tmem_st16(a_addr + h * (G / 4) + 16 * cc, v);
+              unpack_codes32(wst[(hh * (NC / 2) + cc) * kTileN + n], zb, v);
+              tmem_st16(a_addr + slot * AHC + 16 * cc, v);
             }
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {
-              mbar_arrive(&a_full[2 * w + h]);
-              if (h == 1) mbar_arrive(&empty[my_stage]);
+              mbar_arrive(&a_full[w * AH + slot]);
+              if (hh == 1) mbar_arrive(&empty[my_stage]);
             }
           }
           s_p2 = s_p1;
@@ -453,206 +520,176 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
           ++n_pend;
           ++kloc;
         }
+        if (!x_done) x_duty();                           // fewer than AH half-chunks before the segment's end
         if (n_pend == 2) drain(kloc - 2, s_p2);
         if (n_pend >= 1) drain(kloc - 1, s_p1);
         tc_fence_before_sync();
 
-        // ---- end of a tile segment: groups 1..3 hand their accumulators to group 0 -----------
-        if (w != 0) {
+        // ---- end of a tile segment: the four groups' accumulators meet in shared memory; from here
+        //      on warp r owns row r of the tile and lane l its columns 4l..4l+3 ----
 #pragma unroll
-          for (int m = 0; m < MP; ++m) red[((w - 1) * MP + m) * kTileN + n] = acc[m];
-        }
-        named_bar_sync(1, NWG * 128);
-        float acc1[MP];                                 // dual: matrix 1 (up); single: unused
-        if (w == 0) {
-          if (dual) {
-            // even groups hold matrix 0, odd groups matrix 1 (fixed order of the additions)
-#pragma unroll
-            for (int m = 0; m < MP; ++m) {
-              acc[m] += red[(1 * MP + m) * kTileN + n];                                   // group 2
-              acc1[m] = red[(0 * MP + m) * kTileN + n] + red[(2 * MP + m) * kTileN + n];  // groups 1 + 3
-            }
+        for (int m = 0; m < MP; ++m) red[(w * MP + m) * kTileN + n] = acc[m];
+        named_bar_sync(1, kUnpackThreads);
+        const int rw = warp;
+        float f0[4], f1[4] = {0.f, 0.f, 0.f, 0.f};
+        {
+          const float4* r4 = reinterpret_cast<const float4*>(red);
+          const float4 v0 = r4[(0 * MP + rw) * 32 + lane], v1 = r4[(1 * MP + rw) * 32 + lane];
+          const float4 v2 = r4[(2 * MP + rw) * 32 + lane], v3 = r4[(3 * MP + rw) * 32 + lane];
+          if (dual) {                                    // even groups hold matrix 0, odd groups matrix 1
+            f0[0] = v0.x + v2.x; f0[1] = v0.y + v2.y; f0[2] = v0.z + v2.z; f0[3] = v0.w + v2.w;
+            f1[0] = v1.x + v3.x; f1[1] = v1.y + v3.y; f1[2] = v1.z + v3.z; f1[3] = v1.w + v3.w;
           } else {
-#pragma unroll
-            for (int m = 0; m < MP; ++m)
-              acc[m] = ((acc[m] + red[(0 * MP + m) * kTileN + n]) + red[(1 * MP + m) * kTileN + n]) + red[(2 * MP + m) * kTileN + n];
+            f0[0] = ((v0.x + v1.x) + v2.x) + v3.x; f0[1] = ((v0.y + v1.y) + v2.y) + v3.y;
+            f0[2] = ((v0.z + v1.z) + v2.z) + v3.z; f0[3] = ((v0.w + v1.w) + v2.w) + v3.w;
           }
         }
         const bool whole = (g0 == 0 && nch == Gn);
+        const bool finish = (g0 == 0);                   // my run contains the tile's first chunk
         pos += nch;
-        const int my_seg = seg++;
+        const int nmat = dual ? 2 : 1;
 
-        // From here on the tile is handled 4 rows per thread: thread (w, n) owns rows 4w..4w+3 of
-        // column n (both matrices of a dual operation), so that reduction, stores, sums of squares
-        // and arg-max are spread over all 512 unpack threads.
-        float fin[2][4];                                // [matrix][row 4w + r]
-        bool finish = true;
-        if (!whole) {
-          // ---- split tile: every contributor stores its partial and raises a flag (value j + 1);
-          //      the CTA whose run BEGINS the tile adds all partials in CTA order once the flags are
-          //      up.  No atomic read-modify-write, and a CTA only ever waits in its last segment,
-          //      after it has published everything other CTAs need from it (no chain of waits). ----
-          const int my_sl = (my_seg == 0 ? 0 : 1);
-          finish = (g0 == 0);                            // my run contains the tile's first chunk
-          if (w == 0) {
-            float* my = slots + ((size_t)blockIdx.x * 2 + my_sl) * slot_f;
-#pragma unroll
-            for (int m = 0; m < MP; ++m) __stcg(&my[m * kTileN + n], acc[m]);
-            if (dual) {
-#pragma unroll
-              for (int m = 0; m < MP; ++m) __stcg(&my[(MP + m) * kTileN + n], acc1[m]);
-            }
-            if (!finish) {
-              named_bar_sync(2, 128);                    // the group's stores happen-before thread 0's release
-              if (tid == 0) asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(&tile_cnt[blockIdx.x * 2 + my_sl]), "r"(j + 1) : "memory");
-            } else if (tid == 0) {
-              s_flag[1] = (int)op_chunk_owner(op, T * Gn + Gn - 1);   // the last contributor
-            }
+        if (!whole && !finish) {
+          // ---- contributor: (value, tag) pairs, then the flag; no fence in between - the owner
+          //      checks every tag.  (A run that does not begin its tile meets it in its first
+          //      segment, so one slot per CTA is enough.) ----
+          for (int mt = 0; mt < nmat; ++mt) {
+            const float* f = mt ? f1 : f0;
+            uint64_t* dst = my_slot + (size_t)(mt * MP + rw) * kTileN + 4 * lane;
+            st_pairs(dst, tagged(f[0], tag), tagged(f[1], tag));
+            st_pairs(dst + 2, tagged(f[2], tag), tagged(f[3], tag));
           }
-          named_bar_sync(1, NWG * 128);                  // red is free; the finisher's own partial and s_flag are written
-          if (!finish) continue;
-          {
-            const uint32_t first = blockIdx.x, last = (uint32_t)s_flag[1];
-            // wait for the other contributors (thread t polls contributor first + 1 + t); for each of
-            // them this tile is the first segment of its run, i.e. slot 0
-            for (uint32_t i = first + 1 + tid; i <= last; i += NWG * 128)
-              wait_counter(&tile_cnt[i * 2], j + 1, s_abort, sp.ws.status, 9);
-            named_bar_sync(1, NWG * 128);
-            // sums over the contributors in CTA order (the first one is this CTA), loads of up to 8 in flight at once
-            const int nmat = dual ? 2 : 1;
-            for (int mt = 0; mt < nmat; ++mt) {
-              float sum[4] = {0.f, 0.f, 0.f, 0.f};
-              for (uint32_t i0 = first; i0 <= last; i0 += 8) {
-                float v[8][4];
+          named_bar_sync(1, kUnpackThreads);             // red is free; everybody's pairs are on their way
+          if (tid == 0) st_relaxed(&sp.ws.tile_cnt[cta], (int)tag);
+          continue;
+        }
+        if (!whole) {
+          // ---- owner of a split tile: its own partial stays in registers; the others' are added in
+          //      CTA order once their flags are up ----
+          if (tid == 0) s_flag[1] = (int)run_chunk_owner(h.nc, h.cq, h.cr, h.cat_base + T * Gn + Gn - 1);
+          named_bar_sync(1, kUnpackThreads);
+          const uint32_t last = (uint32_t)s_flag[1];
+          for (uint32_t i = cta + 1 + tid; i <= last; i += kUnpackThreads)
+            wait_global<false>(&sp.ws.tile_cnt[i], (int)tag, wc, 10);
+          named_bar_sync(1, kUnpackThreads);
+          const uint64_t* slots64 = reinterpret_cast<const uint64_t*>(sp.ws.slots);
+          for (int mt = 0; mt < nmat; ++mt) {
+            float* f = mt ? f1 : f0;
+            for (uint32_t i0 = cta + 1; i0 <= last; i0 += 2) {
+              uint64_t v[2][4];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                  const uint32_t i = min(i0 + q, last);
-                  const int sl = (i == first) ? my_sl : 0;
-                  const float* src = slots + ((size_t)i * 2 + sl) * slot_f + (size_t)(mt * MP + 4 * w) * kTileN + n;
-#pragma unroll
-                  for (int r = 0; r < 4; ++r) v[q][r] = __ldcg(src + r * kTileN);
-                }
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                  if (i0 + q <= last) {
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) sum[r] += v[q][r];
-                  }
+              for (int q = 0; q < 2; ++q) {
+                const uint32_t i = min(i0 + q, last);
+                const uint64_t* src = slots64 + (size_t)i * kSlotWords + (size_t)(mt * MP + rw) * kTileN + 4 * lane;
+                ld_pairs(src, v[q][0], v[q][1]);
+                ld_pairs(src + 2, v[q][2], v[q][3]);
               }
 #pragma unroll
-              for (int r = 0; r < 4; ++r) fin[mt][r] = sum[r];
+              for (int q = 0; q < 2; ++q) {
+                if (i0 + q > last) continue;
+                bool ok = (uint32_t)(v[q][0] >> 32) == tag && (uint32_t)(v[q][1] >> 32) == tag &&
+                          (uint32_t)(v[q][2] >> 32) == tag && (uint32_t)(v[q][3] >> 32) == tag;
+                if (!ok && !*s_abort) {
+                  // the flag overtook some of the pairs: reload until every tag matches (bounded)
+                  const uint64_t* src = slots64 + (size_t)(i0 + q) * kSlotWords + (size_t)(mt * MP + rw) * kTileN + 4 * lane;
+                  const uint64_t t0 = globaltimer_ns();
+                  while (!ok) {
+                    ld_pairs(src, v[q][0], v[q][1]);
+                    ld_pairs(src + 2, v[q][2], v[q][3]);
+                    ok = (uint32_t)(v[q][0] >> 32) == tag && (uint32_t)(v[q][1] >> 32) == tag &&
+                         (uint32_t)(v[q][2] >> 32) == tag && (uint32_t)(v[q][3] >> 32) == tag;
+                    if (!ok && (*s_abort || globaltimer_ns() - t0 > wc.budget)) { wait_fail(wc, 11); break; }
+                  }
+                }
+#pragma unroll
+                for (int r = 0; r < 4; ++r) f[r] += __uint_as_float((uint32_t)v[q][r]);
+              }
             }
           }
-        } else {
-          // ---- whole tile in this CTA: group 0 redistributes its 16 rows over the four groups ----
-          if (w == 0) {
-#pragma unroll
-            for (int m = 0; m < MP; ++m) {
-              red[m * kTileN + n] = acc[m];
-              if (dual) red[(MP + m) * kTileN + n] = acc1[m];
-            }
-          }
-          named_bar_sync(1, NWG * 128);
-#pragma unroll
-          for (int r = 0; r < 4; ++r) {
-            fin[0][r] = red[(4 * w + r) * kTileN + n];
-            fin[1][r] = dual ? red[(MP + 4 * w + r) * kTileN + n] : 0.f;
-          }
-          named_bar_sync(1, NWG * 128);                  // red is free again
         }
 
-        // ---- tile epilogue, all groups: bf16 stores, sums of squares for the next operation, arg-max ----
-        const int col = (int)T * kTileN + n;
-        float sq[4];
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          const int m = 4 * w + r;
-          const __nv_bfloat16 y0 = __float2bfloat16_rn(fin[0][r]);
-          if (op.out0 != nullptr && m < sp.M) reinterpret_cast<__nv_bfloat16*>(op.out0)[(size_t)m * op.ld_out + col] = y0;
-          float a = __bfloat162float(y0);
+        // ---- tile epilogue: bf16 stores, sums of squares for the next operation, arg-max ----
+        {
+          uint16_t* out0 = ldg_ptr(&op->out0);
+          uint16_t* out1 = ldg_ptr(&op->out1);
+          int32_t* argmax_out = ldg_ptr(&op->argmax_out);
+          const int emit_ssq = __ldg(&op->emit_ssq);
+          const int ld_out = __ldg(&op->ld_out);
+          const int col = (int)T * kTileN + 4 * lane;
+          const bool live = rw < sp.M;
+          float a[4];
+          uint2 y0;
+          y0.x = pack_bf16x2_rn(f0[0], f0[1]);
+          y0.y = pack_bf16x2_rn(f0[2], f0[3]);
+          if (out0 != nullptr && live) *reinterpret_cast<uint2*>(out0 + (size_t)rw * ld_out + col) = y0;
+          a[0] = bf16lo_to_f32(y0.x); a[1] = bf16hi_to_f32(y0.x); a[2] = bf16lo_to_f32(y0.y); a[3] = bf16hi_to_f32(y0.y);
           if (dual) {
-            const __nv_bfloat16 y1 = __float2bfloat16_rn(fin[1][r]);
-            if (m < sp.M) reinterpret_cast<__nv_bfloat16*>(op.out1)[(size_t)m * op.ld_out + col] = y1;
-            if (op.emit_ssq == 2) {
-              a = st_silu(a) * __bfloat162float(y1);
-              if (m < sp.M) __stcg(&sp.ws.act[(size_t)m * op.N + col], a);   // the fp32 product [M][N], for the consumer
+            uint2 y1;
+            y1.x = pack_bf16x2_rn(f1[0], f1[1]);
+            y1.y = pack_bf16x2_rn(f1[2], f1[3]);
+            if (live) *reinterpret_cast<uint2*>(out1 + (size_t)rw * ld_out + col) = y1;
+            if (emit_ssq == 2) {
+              a[0] = st_silu(a[0]) * bf16lo_to_f32(y1.x); a[1] = st_silu(a[1]) * bf16hi_to_f32(y1.x);
+              a[2] = st_silu(a[2]) * bf16lo_to_f32(y1.y); a[3] = st_silu(a[3]) * bf16hi_to_f32(y1.y);
+              // the fp32 product [M][N], for the operation that consumes it
+              if (live) __stcg(reinterpret_cast<float4*>(sp.ws.act + (size_t)rw * __ldg(&op->N) + col), make_float4(a[0], a[1], a[2], a[3]));
             }
           }
-          sq[r] = a * a;
-        }
-        if (op.emit_ssq != 0) {
+          if (emit_ssq != 0) {
+            float sq = ((a[0] * a[0] + a[1] * a[1]) + a[2] * a[2]) + a[3] * a[3];
 #pragma unroll
-          for (int off = 16; off >= 1; off >>= 1)
-#pragma unroll
-            for (int r = 0; r < 4; ++r) sq[r] += __shfl_xor_sync(0xffffffffu, sq[r], off);
-          if (lane == 0) {
-#pragma unroll
-            for (int r = 0; r < 4; ++r) s_part[384 + (4 * w + r) * 4 + wq] = sq[r];
+            for (int off = 16; off >= 1; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
+            if (lane == 0) __stcg(&sp.ws.ssq[((size_t)(j & 1) * sp.ws.n_tiles + T) * 16 + rw], sq);
           }
-        }
-        if (op.argmax_out != nullptr) {
-#pragma unroll
-          for (int r = 0; r < 4; ++r) {
-            float bv = fin[0][r];
+          if (argmax_out != nullptr) {
+            float bv = f0[0];
             int bi = col;
+#pragma unroll
+            for (int r = 1; r < 4; ++r) st_amax_merge(bv, bi, f0[r], col + r);
 #pragma unroll
             for (int off = 16; off >= 1; off >>= 1) {
               const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
               const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
               st_amax_merge(bv, bi, ov, oi);
             }
-            if (lane == 0) s_amax[(4 * w + r) * 4 + wq] = make_float2(bv, __int_as_float(bi));
+            if (lane == 0) __stcg(&sp.ws.cand[(size_t)T * MP + rw], make_float2(bv, __int_as_float(bi)));
           }
-        }
-        named_bar_sync(1, NWG * 128);                    // all stores of the tile issued, per-warp partials in shared memory
-        if (tid < MP) {
-          if (op.emit_ssq != 0) {
-            const float tot = ((s_part[384 + tid * 4] + s_part[384 + tid * 4 + 1]) + s_part[384 + tid * 4 + 2]) + s_part[384 + tid * 4 + 3];
-            __stcg(&sp.ws.ssq[((size_t)(j & 1) * sp.ws.n_tiles + T) * 16 + tid], tot);
-          }
-          if (op.argmax_out != nullptr) {
-            float bv = -INFINITY;
-            int bi = 0x7fffffff;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const float2 c = s_amax[tid * 4 + q];
-              st_amax_merge(bv, bi, c.x, __float_as_int(c.y));
+          named_bar_sync(1, kUnpackThreads);             // all stores of the tile issued; red is free again
+          if (argmax_out != nullptr) {
+            // the CTA that finishes the operation's last tile reduces the per-tile candidates
+            if (tid == 0) {
+              int old;
+              asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(sp.ws.amax_done) : "memory");
+              const int is_last = (old == h.n_tiles - 1);
+              if (is_last) *sp.ws.amax_done = 0;
+              s_flag[3] = is_last;
             }
-            __stcg(&sp.ws.cand[(size_t)T * MP + tid], make_float2(bv, __int_as_float(bi)));
-          }
-        }
-        if (op.argmax_out != nullptr) {
-          // the CTA that finishes the operation's last tile reduces the per-tile candidates
-          named_bar_sync(1, NWG * 128);
-          if (tid == 0) {
-            int old;
-            asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(sp.ws.amax_done) : "memory");
-            const int is_last = (old == op.n_tiles - 1);
-            if (is_last) *sp.ws.amax_done = 0;
-            s_flag[3] = is_last;
-          }
-          named_bar_sync(1, NWG * 128);
-          if (s_flag[3]) {
-            for (int row = warp; row < sp.M; row += NWG * 4) {
-              float bv = -INFINITY;
-              int bi = 0x7fffffff;
-              for (int tt = lane; tt < op.n_tiles; tt += 32) {
-                const float2 c = __ldcg(&sp.ws.cand[(size_t)tt * MP + row]);
-                st_amax_merge(bv, bi, c.x, __float_as_int(c.y));
-              }
+            named_bar_sync(1, kUnpackThreads);
+            if (s_flag[3]) {
+              for (int row = warp; row < sp.M; row += NWG * 4) {
+                float bv = -INFINITY;
+                int bi = 0x7fffffff;
+                for (int tt = lane; tt < h.n_tiles; tt += 32) {
+                  const float2 c = __ldcg(&sp.ws.cand[(size_t)tt * MP + row]);
+                  st_amax_merge(bv, bi, c.x, __float_as_int(c.y));
+                }
 #pragma unroll
-              for (int off = 16; off >= 1; off >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-                const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-                st_amax_merge(bv, bi, ov, oi);
+                for (int off = 16; off >= 1; off >>= 1) {
+                  const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+                  const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+                  st_amax_merge(bv, bi, ov, oi);
+                }
+                if (lane == 0) argmax_out[row] = bi;
               }
-              if (lane == 0) op.argmax_out[row] = bi;
             }
+            named_bar_sync(1, kUnpackThreads);
+          }
+          // the tile is complete: publish it to the operation's counter (one fence after everybody's stores)
+          if (tid == 0 && !(h.flags & kOpNoRelease)) {
+            fence_gpu();
+            red_relaxed_add(&sp.ws.op_done[j], 1);
           }
         }
-        // the tile is complete: publish it to the operation's counter (release after everybody's stores)
-        named_bar_sync(1, NWG * 128);
-        if (tid == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(&sp.ws.op_done[j]) : "memory");
       }
     }
   }
@@ -660,7 +697,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
   // every tensor-memory access of the CTA is complete past this barrier
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == NWG * 4 + 1) {
+  if (warp == kWarpIssuer0) {
     tc_fence_after_sync();
     tmem_dealloc(tmem, TMEM_COLS);
   }
@@ -670,7 +707,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
     const int old = atomicAdd(sp.ws.exit_cnt, 1);
     if (old == (int)gridDim.x - 1) {
       for (int j = 0; j < sp.n_ops; ++j) sp.ws.op_done[j] = 0;
-      for (int i = 0; i < kMaxCtas; ++i) { sp.ws.tile_cnt[i] = 0; sp.ws.tile_cnt[kMaxTiles / 2 + i] = 0; }   // partial-slot flags
+      *sp.ws.amax_done = 0;
       *sp.ws.exit_cnt = 0;
     }
   }
@@ -678,67 +715,50 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
 
 // ---- host side ---------------------------------------------------------------------------------
 
-// Shared-memory plan for a list of operations with common M <= 16 and g; ok = false if some
-// operation's X does not fit beside a ring of at least 4 stages with two CTAs per SM.
+// Shared-memory plan for a list of operations with common M <= 16 and g whose split fields are
+// set; ok = false if some operation's X does not fit beside a ring of at least 6 stages.
 struct StackPlan {
-  int ncta, n_x, n_stages, x_double;
+  int ncta, n_x, n_stages;
   size_t smem;
   bool ok;
 };
 
+int stack_ncta(int sms) { return sms < kMaxCtas / 2 ? sms : kMaxCtas / 2; }   // one 32 KB partial slot per CTA
+
 StackPlan stack_plan(const MegaOp* ops, int n_ops, int g, int sms) {
   StackPlan r = {};
-  int ncta = sms;
-  if (ncta > kMaxCtas / 2) ncta = kMaxCtas / 2;        // two slot sets share the partial-tile region
+  const int ncta = stack_ncta(sms);
   uint32_t n_x = 1;
-  int max_tiles = 1;
-  bool any_indep = false;
   for (int j = 0; j < n_ops; ++j) {
-    const uint32_t per_cta = (ops[j].total_chunks + ncta - 1) / ncta;
-    const uint32_t need = per_cta < (uint32_t)ops[j].n_groups ? per_cta : (uint32_t)ops[j].n_groups;
+    // the longest piece of this operation that one CTA owns
+    uint32_t longest = 0;
+    const uint32_t nc = ops[j].nc;
+    for (uint32_t i = 0; i < nc; ++i) {
+      uint32_t lo, hi;
+      op_local_range(ops[j].nc, ops[j].cq, ops[j].cr, ops[j].cat_base, ops[j].total_chunks, i, lo, hi);
+      if (hi - lo > longest) longest = hi - lo;
+    }
+    const uint32_t need = longest < (uint32_t)ops[j].n_groups ? longest : (uint32_t)ops[j].n_groups;
     if (need > n_x) n_x = need;
-    if (ops[j].n_tiles > max_tiles) max_tiles = ops[j].n_tiles;
-    any_indep = any_indep || ops[j].indep != 0;
   }
-  const uint32_t stage = align128(chunk_bytes(g)), xslot = (uint32_t)MP * 2u * g;
-  const uint32_t fixed = st_fixed_smem() + (uint32_t)n_ops * (uint32_t)sizeof(MegaOp);   // descriptors live in shared memory
-  if (fixed + n_x * xslot + 8 * stage > kStSmemBudget) return r;
-  // a second X buffer lets independent operations overlap; only if it leaves a deep enough ring
-  const bool dbl = any_indep && max_tiles <= kMaxTiles / 2 && fixed + 2 * n_x * xslot + 12 * stage <= kStSmemBudget;
-  r.x_double = dbl ? 1 : 0;
-  const uint32_t xbytes = (dbl ? 2u : 1u) * n_x * xslot;
-  int ns = (int)((kStSmemBudget - fixed - xbytes) / stage);
+  const uint32_t stage = align128(chunk_bytes(g)), xslot = st_xslot_bytes(g);
+  const uint32_t fixed = st_fixed_smem();
+  if (fixed + n_x * xslot + 6 * stage > kStSmemBudget) return r;
+  int ns = (int)((kStSmemBudget - fixed - n_x * xslot) / stage);
   if (ns > kStMaxStages) ns = kStMaxStages;
-  if (const char* e = getenv("QL_STACK_STAGES")) { const int v = atoi(e); if (v >= 2 && v < ns) ns = v; }   // experiments
   r.ncta = ncta; r.n_x = (int)n_x; r.n_stages = ns;
-  r.smem = (size_t)ns * stage + (size_t)xbytes + fixed;
+  r.smem = (size_t)ns * stage + (size_t)n_x * xslot + fixed;
   r.ok = true;
   return r;
 }
 
 template <int G>
 static cudaError_t stack_launch_g(const StackParams& sp, size_t smem, cudaStream_t stream) {
-  static bool attr_set[16] = {};
-  static int max_blocks[16] = {};
-  int dev = 0;
-  cudaGetDevice(&dev);
-  if (dev < 16 && !attr_set[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(qstack_tc5_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(qstack_tc5_kernel<G>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    if (e != cudaSuccess) return e;
-    attr_set[dev] = true;
-  }
   // all CTAs wait on one another's progress: they must be co-resident (the cooperative launch checks it)
-  cudaError_t e = cudaSuccess;
-  int per_sm = 1, sms = sp.ncta;
-  (void)max_blocks;
-  if (getenv("QL_DEBUG")) fprintf(stderr, "[ql] stack launch: ncta %d per_sm %d sms %d smem %zu n_ops %d n_x %d stages %d\n", sp.ncta, per_sm, sms, smem, sp.n_ops, sp.n_x, sp.n_stages);
-  if (per_sm * sms < sp.ncta) return cudaErrorCooperativeLaunchTooLarge;
+  cudaError_t e = cudaFuncSetAttribute(qstack_tc5_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStSmemBudget);
+  if (e != cudaSuccess) return e;
   void* args[] = {const_cast<StackParams*>(&sp)};
-  e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(qstack_tc5_kernel<G>), dim3(sp.ncta), dim3(kStThreads), args, smem, stream);
-  if (e != cudaSuccess && getenv("QL_DEBUG")) fprintf(stderr, "[ql] stack launch failed: %s\n", cudaGetErrorString(e));
-  return e;
+  return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(qstack_tc5_kernel<G>), dim3(sp.ncta), dim3(kStThreads), args, smem, stream);
 }
 
 cudaError_t launch_stack_tc5(const StackParams& sp, int g, size_t smem, cudaStream_t stream) {

@@ -51,7 +51,7 @@ def test_size_queries(pkg):
     assert pkg.ql_workspace_bytes(64, 151936) >= pkg.ql_workspace_bytes(16, 151936)
     assert pkg.ql_workspace_bytes(0, 128) == 0 and pkg.ql_workspace_bytes(65, 128) == 0
     assert pkg.ql_workspace_bytes(16, 100) == 0
-    assert pkg.ql_select_path(16, 2560, 9728, 128) in (pkg.QL_PATH_FMA, pkg.QL_PATH_MMA, pkg.QL_PATH_TC5)
+    assert pkg.ql_select_path(16, 2560, 9728, 128) in (pkg.QL_PATH_MMA, pkg.QL_PATH_TC5)
     assert pkg.ql_select_path(16, 2560, 9728, 96) < 0
 
 

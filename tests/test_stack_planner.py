@@ -1,6 +1,6 @@
 """Host logic of the stack launcher, without a GPU: which operations are fused into the persistent
-kernel, which gate/up pairs become dual operations, which glue operations are folded, which
-operations may skip their predecessor's dependency wait, and what falls back to single launches.
+kernel, which gate/up pairs become dual operations, which glue operations are folded, which runs
+are independent linears streamed as one piece per thread block, and what falls back to single launches.
 Pointers are fake (never dereferenced: ql_stack_plan launches nothing)."""
 import pytest
 
@@ -61,7 +61,8 @@ def test_gate_up_without_their_glue_stay_two_operations(ql):
     ops = layer_ops(0)[4:6]                      # gate, up only
     c = plan(ql, ops)
     assert c["fused_ops"] == 2 and c["dual_ops"] == 0
-    assert c["independent"] == 1                 # up shares no buffer with gate except the input both read
+    # up shares no buffer with gate except the input both read: the two run as one stream of chunks
+    assert c["independent"] == 1 and c["batch_launches"] == 1
 
 
 def test_independent_linears_skip_the_wait_but_write_after_write_does_not(ql):
@@ -71,9 +72,14 @@ def test_independent_linears_skip_the_wait_but_write_after_write_does_not(ql):
     assert c["fused_ops"] == 6 and c["independent"] == 5 and c["batch_launches"] == 1
     c = plan(ql, [lin(i, buf(20)) for i in range(6)])          # same output buffer: ordered
     assert c["independent"] == 0 and c["batch_launches"] == 0
-    # independent of the neighbour but not pairwise (ops 0 and 2 write the same buffer): no batch kernel
+    # independent of the neighbour but not pairwise (ops 0 and 2 write the same buffer): a chain
     c = plan(ql, [lin(0, buf(20)), lin(1, buf(21)), lin(2, buf(20))])
-    assert c["independent"] == 2 and c["batch_launches"] == 0
+    assert c["independent"] == 0 and c["batch_launches"] == 0
+    # K of more than 24 groups: the X of a whole operation would not fit in shared memory, so a chain
+    def wide(i):
+        return dict(kind=0, M=16, K=9728, N=2560, g=128, ld_in=9728, ld_out=2560, packed=buf(100 + i), in0=buf(1), out=buf(20 + i))
+    c = plan(ql, [wide(i) for i in range(4)])
+    assert c["fused_ops"] == 4 and c["batch_launches"] == 0 and c["independent"] == 0
     # a linear that reads its predecessor's output is dependent
     a = dict(kind=0, M=16, K=2560, N=2560, g=128, ld_in=2560, ld_out=2560, packed=buf(100), in0=buf(1), out=buf(2))
     b = dict(kind=0, M=16, K=2560, N=2560, g=128, ld_in=2560, ld_out=2560, packed=buf(101), in0=buf(2), out=buf(3))
