@@ -140,6 +140,14 @@ int qlinear_w4a16_path(const void* packed, const uint16_t* X, uint16_t* Y, int32
 /* The path qlinear_w4a16 takes for a shape (a ql_path other than AUTO), or a negative ql_status. */
 int ql_select_path(int M, int K, int N, int g);
 
+/* How a linear launched on its own would be set up, without launching (needs no device: it then
+ * plans for 148 SMs).  out (HOST, 4 ints): [0] the path taken (path == QL_PATH_AUTO: the selected
+ * one), and for the warp-level MMA path [1] the depth of the shared-memory ring, [2] the groups of
+ * X held in shared memory per thread block, [3] 0 if the X columns a block needs stay resident,
+ * else the number of chunks after which they are reloaded (large M with long K).
+ * Errors: QL_ERR_NULL, QL_ERR_SHAPE, QL_ERR_UNSUPPORTED. */
+int ql_linear_plan(int M, int K, int N, int g, int path, int out[4]);
+
 /*
  * qlinear_stack_w4a16 - run a list of operations in order on one stream: the projections of one
  * or many decoder layers (q/k/v/o, gate/up/down) and the LM head of one verify step (Section 2.2:
@@ -253,6 +261,28 @@ uint32_t ql_plan_chunk_owner(uint32_t total_chunks, uint32_t ncta, uint32_t chun
  * runs to its end without hanging; -1 switches the hook off.  Nothing traps or faults. */
 void ql_debug_set_wait_budget_ns(uint64_t ns);
 void ql_debug_no_release(int fused_op);
+
+/* In-kernel timeline of the persistent kernel, for builds of the library with -DQL_TIMELINE
+ * (ql_debug_timeline_enabled() == 1; the regular build compiles the stamps out and returns 0).
+ * ql_debug_set_timeline(buf): launches that follow write globaltimer stamps (ns) into the DEVICE
+ * buffer: first [160 thread blocks][n_ops][16] SM cycle stamps of thread 0 (0 operation entered,
+ * 1 first chunk unpacked, 2 predecessor known complete, 3 X operand built, 4-6 first tile segment
+ * drained / exchanged / published, 7 the watcher saw the predecessor complete, 8-14 the same
+ * steps of the last tile segment incl. 10 contributors' flags seen, 11 partials added, 12 stores
+ * issued, 14 published, 15 the publish time in globaltimer ns), then [160][4][8] cycle sums of the
+ * unpack groups, [160][4][8] of the MMA issuers, and [160][n_ops] globaltimer ns at which the
+ * watcher saw the predecessor complete.  paper_2607_04244_b200/timeline.py sizes and reads it.
+ * NULL switches the stamps off. */
+void ql_debug_set_timeline(void* device_buffer);
+int ql_debug_timeline_enabled(void);
+
+/* Timing experiments on the persistent kernel: launches that follow leave out the phases named by
+ * `mask` (1 weight copies, unpacking and MMAs; 2 loading and converting the X operand; 4 waiting for
+ * the row scales; 8 the exchange of split tiles; 16 the fence before a row is published; 32 the
+ * accumulator exchange through shared memory; 64 the row epilogue; 256 the watcher's acquire
+ * fence).  The RESULTS ARE GARBAGE while mask != 0; the step time that remains tells what the
+ * left-out phases cost on the critical path.  0 restores normal operation. */
+void ql_debug_set_ablate(int mask);
 
 /* Number of kernels the library has launched since it was loaded (all entry points, this
  * process).  For benchmarks that report their launch count. */

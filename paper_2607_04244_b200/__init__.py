@@ -23,8 +23,8 @@ EXPORTS = [
     "ql_status_str", "ql_packed_bytes", "ql_workspace_bytes", "ql_workspace_init", "ql_device_status",
     "ql_device_status_raw",
     "qpack_w4_g128", "qlinear_w4a16", "qlinear_w4a16_path", "ql_select_path", "qlinear_stack_w4a16",
-    "qlinear_stack_w4a16_host", "ql_launch_count", "qlinear_w4a16_static", "ql_static_status", "ql_stack_plan", "ql_plan_first_chunk", "ql_plan_chunk_owner",
-    "ql_debug_set_wait_budget_ns", "ql_debug_no_release",
+    "qlinear_stack_w4a16_host", "ql_launch_count", "qlinear_w4a16_static", "ql_static_status", "ql_stack_plan", "ql_linear_plan", "ql_plan_first_chunk", "ql_plan_chunk_owner",
+    "ql_debug_set_wait_budget_ns", "ql_debug_no_release", "ql_debug_set_timeline", "ql_debug_timeline_enabled", "ql_debug_set_ablate",
 ]
 
 
@@ -88,6 +88,8 @@ def load(path: str | None = None):
     lib.ql_static_status.argtypes = [ctypes.POINTER(ctypes.c_int), vp]
     lib.ql_stack_plan.restype = i32
     lib.ql_stack_plan.argtypes = [ctypes.POINTER(ql_op), i32, vp, sz, ctypes.POINTER(ctypes.c_int)]
+    lib.ql_linear_plan.restype = i32
+    lib.ql_linear_plan.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(ctypes.c_int)]
     for fn in (lib.ql_plan_first_chunk, lib.ql_plan_chunk_owner):
         fn.restype = ctypes.c_uint32
         fn.argtypes = [ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32]
@@ -95,6 +97,12 @@ def load(path: str | None = None):
     lib.ql_debug_set_wait_budget_ns.argtypes = [ctypes.c_uint64]
     lib.ql_debug_no_release.restype = None
     lib.ql_debug_no_release.argtypes = [i32]
+    lib.ql_debug_set_timeline.restype = None
+    lib.ql_debug_set_timeline.argtypes = [vp]
+    lib.ql_debug_set_ablate.restype = None
+    lib.ql_debug_set_ablate.argtypes = [i32]
+    lib.ql_debug_timeline_enabled.restype = i32
+    lib.ql_debug_timeline_enabled.argtypes = []
     lib.ql_launch_count.restype = ctypes.c_uint64
     lib.ql_launch_count.argtypes = []
     _lib = lib
@@ -140,6 +148,19 @@ def ql_debug_set_wait_budget_ns(ns: int) -> None:
 
 def ql_debug_no_release(fused_op: int) -> None:
     load().ql_debug_no_release(fused_op)
+
+
+def ql_debug_set_timeline(buf) -> None:
+    """buf: an int64 device tensor of at least 160 * n_ops * 8 elements, or None."""
+    load().ql_debug_set_timeline(None if buf is None else buf.data_ptr())
+
+
+def ql_debug_set_ablate(mask: int) -> None:
+    load().ql_debug_set_ablate(mask)
+
+
+def ql_debug_timeline_enabled() -> bool:
+    return bool(load().ql_debug_timeline_enabled())
 
 
 # ---- device entry points ----------------------------------------------------------------------
@@ -232,6 +253,13 @@ def ql_static_status(stream=None) -> int:
     out = ctypes.c_int(-1)
     _check(load().ql_static_status(ctypes.byref(out), _stream(stream)), "ql_static_status")
     return out.value
+
+
+def ql_linear_plan(M: int, K: int, N: int, g: int, path: int = QL_PATH_AUTO) -> dict:
+    """How qlinear_w4a16 would set up this linear (no launch, no device needed)."""
+    c = (ctypes.c_int * 4)()
+    _check(load().ql_linear_plan(M, K, N, g, path, c), "ql_linear_plan")
+    return dict(zip(["path", "n_stages", "n_x", "x_phase"], list(c)))
 
 
 def ql_stack_plan(ops, ws_ptr: int, ws_bytes: int) -> dict:

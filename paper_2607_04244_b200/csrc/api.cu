@@ -10,6 +10,7 @@
 namespace ql {
 cudaError_t launch_qpack(const uint32_t*, const uint16_t*, const uint8_t*, int, int, int, uint8_t*, cudaStream_t);
 cudaError_t launch_linear_mma(LinearParams, cudaStream_t);
+size_t plan_linear_mma(LinearParams&);
 cudaError_t launch_linear_tc5(LinearParams, int sms, cudaStream_t, bool pdl);
 bool tc5_supported(const LinearParams&, int sms);
 struct StackPlan { int ncta, n_x, n_stages; size_t smem; bool ok; };
@@ -22,6 +23,8 @@ static std::atomic<uint64_t> g_launches{0};
 static std::atomic<uint32_t> g_epoch{0};                  // stack-kernel launches: tags of split-K partial tiles
 static std::atomic<uint64_t> g_wait_ns{kWaitBudgetNs};    // budget of the stack kernel's bounded waits
 static std::atomic<int> g_no_release_op{-1};              // test hook: fused operation that does not publish its tiles
+static std::atomic<int> g_ablate{0};                      // timing experiments: phases of the stack kernel switched off
+static std::atomic<uint64_t*> g_timeline{nullptr};        // device buffer for the in-kernel timeline (QL_TIMELINE builds)
 
 static bool shape_ok(int M, int K, int N, int g) {
   if (M < 1 || M > 64) return false;
@@ -187,17 +190,21 @@ static bool independent_ops(const MegaOp& prev, const MegaOp& cur, int M) {
 constexpr int kBatchMaxGroups = 24;   // K <= 24 groups: X of one operation (24 x 4.25 KB) beside a useful ring
 
 // True if the run is a list of plain linears no two of which share a buffer other than inputs
-// that both only read: such a run goes to the batch kernel, which overlaps its operations freely.
-static bool batchable(const std::vector<MegaOp>& mega, int M) {
+// that both only read: nothing in it has to wait for a result.
+static bool independent_run(const std::vector<MegaOp>& mega, int M) {
   if (mega.size() < 2) return false;
   for (const MegaOp& m : mega)
     if (m.packed1 != nullptr || m.prologue != 0 || m.emit_ssq != 0 || m.argmax_out != nullptr || m.out0 == nullptr) return false;
-  // one CTA works through a long piece of the run: the X of a whole operation has to fit in shared memory
-  for (const MegaOp& m : mega)
-    if (m.n_groups > kBatchMaxGroups) return false;
   for (size_t a = 0; a < mega.size(); ++a)
     for (size_t b = a + 1; b < mega.size(); ++b)
       if (!independent_ops(mega[a], mega[b], M) || !independent_ops(mega[b], mega[a], M)) return false;
+  return true;
+}
+// An independent run is laid end to end and cut into one piece per CTA if the X of a whole
+// operation fits in shared memory (a piece spans whole tile columns).
+static bool fits_one_stream(const std::vector<MegaOp>& mega) {
+  for (const MegaOp& m : mega)
+    if (m.n_groups > kBatchMaxGroups) return false;
   return true;
 }
 
@@ -212,7 +219,7 @@ static bool is_dual(const ql_op* ops, int i, int n_ops) {
 }
 
 // Operations per stack-kernel launch (the partial-tile tags keep 9 bits for the operation number).
-constexpr int kStackRunOps = 256;
+constexpr int kStackRunOps = kMaxOps;
 
 // What the planner made of an operation list (ql_stack_plan reports it without launching).
 struct StackCounts {
@@ -246,7 +253,8 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
       // Independent plain linears form ONE run: their chunks are laid end to end and every CTA
       // takes one contiguous piece.  Anything else is a chain: every operation is its own run and
       // waits for the one before it.
-      const bool batch = batchable(mega, run_M);
+      const bool indep = independent_run(mega, run_M);
+      const bool batch = indep && fits_one_stream(mega);
       if (batch) {
         uint32_t total = 0;
         for (MegaOp& m : mega) { m.cat_base = total; total += m.total_chunks; }
@@ -256,7 +264,10 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
           MegaOp& m = mega[j];
           m.cat_base = 0;
           run_split(m.total_chunks, (uint32_t)ncta, m.nc, m.cq, m.cr);
-          if (j > 0) m.flags |= kOpWait;
+          // independent operations whose K is too long for one stream: each is split among all CTAs
+          // like a chained one, but waits only for the operation two back
+          if (indep) { if (j > 1) m.flags |= kOpWait2; }
+          else if (j > 0) m.flags |= kOpWait;
         }
       }
       const int hook = g_no_release_op.load(std::memory_order_relaxed);
@@ -270,6 +281,8 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
       sp.ops = reinterpret_cast<const MegaOp*>(sp.ws.desc);
       sp.n_ops = (int)mega.size(); sp.M = run_M; sp.ncta = plan.ncta; sp.n_stages = plan.n_stages; sp.n_x = plan.n_x;
       sp.wait_ns = g_wait_ns.load(std::memory_order_relaxed);
+      sp.ablate = g_ablate.load(std::memory_order_relaxed);
+      sp.timeline = g_timeline.load(std::memory_order_relaxed);
       cnt.stack_launches += 1;
       cnt.batch_launches += batch ? 1 : 0;
       cnt.fused_ops += (int)mega.size();
@@ -467,6 +480,30 @@ int ql_select_path(int M, int K, int N, int g) {
   return select_path(p, sms);
 }
 
+int ql_linear_plan(int M, int K, int N, int g, int path, int out[4]) {
+  if (out == nullptr) return QL_ERR_NULL;
+  if (!shape_ok(M, K, N, g)) return QL_ERR_SHAPE;
+  if (path != QL_PATH_AUTO && path != QL_PATH_MMA && path != QL_PATH_TC5) return QL_ERR_UNSUPPORTED;
+  LinearParams p = {};
+  p.M = M; p.K = K; p.N = N; p.g = g;
+  p.n_tiles = N / kTileN; p.n_groups = K / g;
+  p.total_chunks = (uint32_t)p.n_tiles * (uint32_t)p.n_groups;
+  int sms = num_sms();
+  if (sms <= 0) sms = 148;                              // no device: answer for a B200
+  int ncta = sms < kMaxCtas ? sms : kMaxCtas;
+  if ((uint32_t)ncta > p.total_chunks) ncta = (int)p.total_chunks;
+  p.ncta = ncta;
+  p.m_pad = pad_rows(M);
+  if (path == QL_PATH_AUTO) path = select_path(p, sms);
+  if (path == QL_PATH_TC5 && !tc5_supported(p, sms)) return QL_ERR_UNSUPPORTED;
+  out[0] = path; out[1] = 0; out[2] = 0; out[3] = 0;
+  if (path == QL_PATH_MMA) {
+    if (plan_linear_mma(p) == 0) return QL_ERR_UNSUPPORTED;
+    out[1] = p.n_stages; out[2] = p.n_x; out[3] = p.x_phase;
+  }
+  return QL_OK;
+}
+
 int qlinear_w4a16_path(const void* packed, const uint16_t* X, uint16_t* Y, int32_t* argmax_out, int M, int K, int N,
                        int g, void* workspace, size_t workspace_bytes, void* stream, int path) {
   LinearParams p;
@@ -554,6 +591,15 @@ uint32_t ql_plan_chunk_owner(uint32_t total_chunks, uint32_t ncta, uint32_t chun
 }
 
 void ql_debug_set_wait_budget_ns(uint64_t ns) { g_wait_ns.store(ns == 0 ? kWaitBudgetNs : ns, std::memory_order_relaxed); }
+void ql_debug_set_timeline(void* device_buffer) { g_timeline.store(static_cast<uint64_t*>(device_buffer), std::memory_order_relaxed); }
+int ql_debug_timeline_enabled(void) {
+#ifdef QL_TIMELINE
+  return 1;
+#else
+  return 0;
+#endif
+}
+void ql_debug_set_ablate(int mask) { g_ablate.store(mask, std::memory_order_relaxed); }
 void ql_debug_no_release(int fused_op) { g_no_release_op.store(fused_op, std::memory_order_relaxed); }
 
 uint64_t ql_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

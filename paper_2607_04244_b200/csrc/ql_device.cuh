@@ -15,9 +15,11 @@ __host__ __device__ constexpr uint32_t align128(uint32_t x) { return (x + 127u) 
 
 // ---- workspace layout -----------------------------------------------------------------------
 // [0, 256)        control header: word 0 status, word 1 finished-tile counter (arg-max),
-//                 word 2 finished-CTA counter of the stack kernel
-// then            per-tile arrival counters (split-K)            [kMaxTiles]
-// then            per-operation finished-tile counters (stack)   [kMaxOps]
+//                 word 2 finished-CTA counter of the stack kernel, words 16-31 its per-row arg-max counters
+// then            per-tile arrival counters (split-K) of the single-linear kernels / partial-row flags of
+//                 the stack kernel                               [kFlagWords]
+// then            per-operation, per-row finished-tile counters of the stack kernel, one 128-byte line each
+//                                                                [kMaxOps][16][32]
 // -- everything above is zero between calls (ql_workspace_init zeroes it once, kernels restore it) --
 // then            operation descriptors of the stack kernel      [kMaxOps * kOpDescBytes]
 // then            row sums of squares per tile, two buffers      [2][tiles][16] fp32
@@ -26,10 +28,12 @@ __host__ __device__ constexpr uint32_t align128(uint32_t x) { return (x + 127u) 
 // then            split-K partial tiles  [kMaxCtas][2 segments][2 matrices][m_pad*128] fp32
 constexpr int kMaxCtas = 320;                     // up to two CTAs per SM
 constexpr int kMaxTiles = 4096;                   // N <= 128 * 4096
-constexpr int kMaxOps = 1024;                     // fused operations per stack-kernel launch
+constexpr int kFlagWords = 8192;                  // tile counters / partial-row flags: [2 parities][160 CTAs][16 rows] fit
+constexpr int kMaxOps = 256;                      // fused operations per stack-kernel launch
+constexpr int kOpDoneStride = 32;                 // ints between the counters of two rows (one line each: they are polled)
 constexpr int kOpDescBytes = 128;
 constexpr int kWsHeaderBytes = 256;
-constexpr size_t kWsControlBytes = kWsHeaderBytes + (size_t)kMaxTiles * 4 + (size_t)kMaxOps * 4;
+constexpr size_t kWsControlBytes = kWsHeaderBytes + (size_t)kFlagWords * 4 + (size_t)kMaxOps * 16 * kOpDoneStride * 4;
 constexpr size_t kWsDescBytes = (size_t)kMaxOps * kOpDescBytes;
 
 struct Workspace {
@@ -66,7 +70,7 @@ __host__ __device__ inline Workspace ws_carve(void* base, int n_tiles, int m_pad
   w.amax_done = (int*)p + 1;
   w.exit_cnt = (int*)p + 2;
   w.tile_cnt = (int*)(p + kWsHeaderBytes);
-  w.op_done = w.tile_cnt + kMaxTiles;
+  w.op_done = w.tile_cnt + kFlagWords;
   w.desc = (uint8_t*)(p + kWsControlBytes);
   p += kWsControlBytes + kWsDescBytes;
   w.ssq = (float*)p;

@@ -35,6 +35,7 @@ struct LinearParams {
 // The first 32 bytes hold what every role reads at every operation.
 constexpr int kOpDual = 1;        // two matrices (packed0, packed1) share X
 constexpr int kOpWait = 2;        // X may be read only after operation j-1 has finished every tile
+constexpr int kOpWait2 = 8;       // X may be read only after operation j-2 has finished (its partial-tile slots are reused)
 constexpr int kOpNoRelease = 4;   // test hook: finished tiles are not published (the next operation's wait runs out)
 struct MegaOp {
   uint32_t nc, cq, cr;     // CTA i owns run positions [i*cq + i*cr/nc, (i+1)*cq + (i+1)*cr/nc), i < nc
@@ -65,8 +66,10 @@ struct StackParams {
   int ncta;
   int n_stages;            // ring depth
   int n_x;                 // X slots (groups) in shared memory
+  int ablate;              // timing experiments only (see the stack kernel); 0 in production
   uint32_t epoch;          // launch number: partial tiles in the workspace carry (epoch, operation) tags
   uint64_t wait_ns;        // budget of every bounded wait
+  uint64_t* timeline;      // builds with -DQL_TIMELINE only: [ncta][n_ops][8] globaltimer stamps, else nullptr
   Workspace ws;
 };
 

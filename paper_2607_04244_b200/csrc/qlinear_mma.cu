@@ -374,8 +374,9 @@ static cudaError_t launch_one(const LinearParams& p, size_t smem, cudaStream_t s
   return cudaGetLastError();
 }
 
-// Fills the path-specific fields of `p` and launches.  Returns a cudaError_t.
-cudaError_t launch_linear_mma(LinearParams p, cudaStream_t stream) {
+// Fills the path-specific fields of `p` (ring depth, X slots, resident or phased X); returns the
+// dynamic shared memory the launch needs, 0 if the shape cannot run.
+size_t plan_linear_mma(LinearParams& p) {
   const int mt = p.m_pad / 16;
   const int mtt = mt <= 1 ? 1 : (mt == 2 ? 2 : 4);           // kernels exist for 16, 32 and 64 padded rows
   p.m_pad = mtt * 16;
@@ -389,7 +390,7 @@ cudaError_t launch_linear_mma(LinearParams p, cudaStream_t stream) {
   if (fixed + (uint32_t)p.n_x * xslot + min_ring > kSmemBudget) {
     // X of all the CTA's groups does not fit beside a useful ring: reload it every x_phase chunks
     const int fit = (int)((kSmemBudget - fixed - min_ring) / xslot);
-    if (fit < 1) return cudaErrorInvalidConfiguration;
+    if (fit < 1) return 0;
     p.n_x = fit;
     p.x_phase = fit;
   }
@@ -399,7 +400,14 @@ cudaError_t launch_linear_mma(LinearParams p, cudaStream_t stream) {
   if ((uint32_t)ns > per_cta) ns = (int)per_cta;
   if (ns < 2) ns = 2;
   p.n_stages = ns;
-  const size_t smem = (size_t)ns * p.stage_bytes + xbytes + fixed;
+  return (size_t)ns * p.stage_bytes + xbytes + fixed;
+}
+
+// Fills the path-specific fields of `p` and launches.  Returns a cudaError_t.
+cudaError_t launch_linear_mma(LinearParams p, cudaStream_t stream) {
+  const size_t smem = plan_linear_mma(p);
+  if (smem == 0) return cudaErrorInvalidConfiguration;
+  const int mtt = p.m_pad / 16;
   if (p.g == 128) {
     if (mtt == 1) return launch_one<1, 128>(p, smem, stream);
     if (mtt == 2) return launch_one<2, 128>(p, smem, stream);

@@ -72,7 +72,7 @@ extern "C" int qlinear_w4a16_static(const void* packed, const uint16_t* X, uint1
   w.amax_done = w.status + 1;
   w.exit_cnt = w.status + 2;
   w.tile_cnt = reinterpret_cast<int*>(scratch + kWsHeaderBytes);
-  w.op_done = w.tile_cnt + kMaxTiles;
+  w.op_done = w.tile_cnt + kFlagWords;
   w.cand = reinterpret_cast<float2*>(scratch + kWsControlBytes);
   w.slots = reinterpret_cast<float*>(scratch + kWsControlBytes + kStaticCandBytes);
   w.n_tiles = kStaticMaxTiles;

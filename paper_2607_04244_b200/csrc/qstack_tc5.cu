@@ -11,7 +11,8 @@
 //   16     producer: one bulk copy (TMA engine, no tensor map, no multicast) per packed chunk into a
 //          ring of shared-memory stages; it runs ahead over operation boundaries, so the weights of
 //          operation j+1 are on chip while operation j is still being reduced.
-//   17-20  one MMA issuer per unpack group (a tcgen05.mma costs its issuing thread ~50-150 cycles).
+//   17-20  one MMA issuer per unpack group (a tcgen05.mma with N = 16 costs its issuing thread
+//          ~150 cycles while tensor-memory stores are running, and a chunk needs 8).
 //   21     watcher: polls the counter of the previous operation, so that the other warps can work
 //          while they wait, and computes the row scales 1/rms from the per-tile sums of squares.
 //
@@ -21,10 +22,12 @@
 //     the issuers hold the MMAs back until X has been published;
 //   * waiting is done with relaxed loads (no fence per poll); the one acquire fence follows the
 //     successful poll;
-//   * split tiles: a contributor writes its partial sums as (value, tag) pairs and then sets a
-//     flag without a fence in between; the owner of the tile polls the flag, loads the pairs and
-//     checks every tag (a pair is one 8-byte store, so a matching tag proves the value), adding them
-//     in CTA order - deterministic, no floating-point atomics;
+//   * the end of a tile is handled row by row: after one exchange through shared memory warp r owns
+//     row r, and from there on the 16 warps never meet again - a contributor's warp stores its row
+//     of the partial tile, fences and raises the row's flag (tagged with launch and operation
+//     number, so flags are never reset); the owner's warp r polls the contributors' row flags, adds
+//     their rows in CTA order (deterministic, no floating-point atomics), stores the bf16 row and the
+//     row's sum of squares and publishes the row to a per-row counter of the operation;
 //   * the glue between linears is folded in: a finished tile also leaves the row sums of squares
 //     of what the next operation normalises, and that operation builds its X operand as
 //     bf16(in * rsqrt(mean square)) (optionally of silu(gate) * up) while it loads it;
@@ -41,16 +44,18 @@ constexpr int NWG = 4;                                  // unpack groups per CTA
 constexpr int AH = 3;                                   // half-chunk A buffers per group
 constexpr int MP = 16;                                  // padded rows
 constexpr int kUnpackThreads = NWG * 128;               // 512
-constexpr int kWarpProducer = NWG * 4, kWarpIssuer0 = NWG * 4 + 1, kWarpWatcher = NWG * 4 + 1 + NWG;
+constexpr int kIssuers = NWG;                           // one per group
+constexpr int kWarpProducer = NWG * 4, kWarpIssuer0 = NWG * 4 + 1, kWarpWatcher = NWG * 4 + 1 + kIssuers;
 constexpr int kStThreads = (kWarpWatcher + 1) * 32;     // 704
 constexpr int kStMaxStages = 24;
 constexpr uint32_t kStSmemBudget = 232448u;
 constexpr uint32_t kXLbo = 16u * MP + 16u;              // bytes between K-adjacent 8x16-byte core matrices (+16: bank spread)
 __host__ __device__ constexpr uint32_t st_xslot_bytes(int g) { return (uint32_t)(g / 8) * kXLbo; }
-__host__ __device__ constexpr uint32_t st_fixed_smem() { return NWG * MP * 128u * 4u + 1024u; }
-constexpr uint32_t kSlotWords = 2u * MP * 128u;         // (value, tag) pairs of one CTA's partial tile, two matrices
+// accumulator exchange buffer + barriers, flags and the two descriptor slots (656 + 64 + 128 + 256 bytes)
+__host__ __device__ constexpr uint32_t st_fixed_smem() { return NWG * MP * 128u * 4u + 2048u; }
+constexpr uint32_t kSlotWords = 2u * MP * 128u;         // floats of one CTA's partial tile, two matrices
 
-__device__ __forceinline__ float st_silu(float v) { return v / (1.f + __expf(-v)); }
+__device__ __forceinline__ float st_silu(float v) { return __fdividef(v, 1.f + __expf(-v)); }
 __device__ __forceinline__ void st_amax_merge(float& bv, int& bi, float v, int i) {
   if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
 }
@@ -66,14 +71,48 @@ __device__ __forceinline__ void red_relaxed_add(int* p, int v) {
   asm volatile("red.relaxed.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void fence_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
-__device__ __forceinline__ void ld_pairs(const uint64_t* p, uint64_t& a, uint64_t& b) {
-  asm volatile("ld.relaxed.gpu.global.v2.b64 {%0,%1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
-}
-__device__ __forceinline__ void st_pairs(uint64_t* p, uint64_t a, uint64_t b) {
-  asm volatile("st.relaxed.gpu.global.v2.b64 [%0], {%1,%2};" ::"l"(p), "l"(a), "l"(b) : "memory");
-}
-__device__ __forceinline__ uint64_t tagged(float v, uint32_t tag) { return ((uint64_t)tag << 32) | (uint64_t)__float_as_uint(v); }
 
+// In-kernel timeline (builds with -DQL_TIMELINE): thread 0 of a CTA stamps the phases of every
+// operation, the watcher's lane 0 the moment it saw the previous operation complete.
+// slots: 0 operation entered, 1 first chunk unpacked (before X), 2 dependency seen, 3 X built,
+//        4 last chunk of the first segment drained, 5 its accumulators exchanged, 6 its tile published / partial sent,
+//        7 watcher saw the predecessor complete; of the LAST segment: 8 drained, 9 exchanged, 10 contributors' flags
+//        seen, 11 partials added, 12 epilogue stores issued, 13 barrier passed, 14 published / partial sent
+#ifdef QL_TIMELINE
+// (stamps are SM cycle counts, comparable within a thread block; slots 7 and 15 also exist as globaltimer
+//  nanoseconds, 256 ns resolution, in a second array for comparisons between thread blocks)
+#define QL_STAMP(slot) do { if (sp.timeline != nullptr && tid == 0) { sp.timeline[((size_t)cta * sp.n_ops + j) * 16 + (slot)] = (uint64_t)clock64(); \
+    if ((slot) == 14) sp.timeline[((size_t)cta * sp.n_ops + j) * 16 + 15] = globaltimer_ns(); } } while (0)
+#define QL_STAMP_W(slot) do { if (sp.timeline != nullptr && lane == 0) { sp.timeline[((size_t)cta * sp.n_ops + j) * 16 + (slot)] = (uint64_t)clock64(); \
+    sp.timeline[(size_t)160 * sp.n_ops * 16 + (size_t)2 * 160 * NWG * 8 + (size_t)cta * sp.n_ops + j] = globaltimer_ns(); } } while (0)
+// cycle accounting of the unpack loop (lane 0 of the first warp of every group):
+// 0 wait for the ring stage, 1 wait for a free A buffer, 2 unpack + tensor-memory stores issued, 3 wait::st,
+// 4 wait for the MMAs of the chunk two back, 5 tensor-memory load + scale-accumulate, 6 chunks
+#define QL_CYC_DECL long long cyc_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long cyc_t_ = 0; (void)cyc_t_
+#define QL_CYC_BEGIN() do { cyc_t_ = clock64(); } while (0)
+#define QL_CYC_END(i) do { const long long now_ = clock64(); cyc_[i] += now_ - cyc_t_; cyc_t_ = now_; } while (0)
+#define QL_CYC_ADD(i, v) do { cyc_[i] += (v); } while (0)
+#define QL_CYC_FLUSH() do { if (sp.timeline != nullptr && wq == 0 && lane == 0) { \
+    uint64_t* dst_ = sp.timeline + (size_t)160 * sp.n_ops * 16 + ((size_t)cta * NWG + w) * 8; \
+    for (int i_ = 0; i_ < 8; ++i_) dst_[i_] = (uint64_t)cyc_[i_]; } } while (0)
+#define QL_CYC_FLUSH_I() do { if (sp.timeline != nullptr) { \
+    uint64_t* dst_ = sp.timeline + (size_t)160 * sp.n_ops * 16 + (size_t)160 * NWG * 8 + ((size_t)cta * NWG + w) * 8; \
+    for (int i_ = 0; i_ < 8; ++i_) dst_[i_] = (uint64_t)cyc_[i_]; } } while (0)
+#else
+#define QL_CYC_FLUSH_I() do {} while (0)
+#define QL_STAMP(slot) do {} while (0)
+#define QL_STAMP_W(slot) do {} while (0)
+#define QL_CYC_DECL do {} while (0)
+#define QL_CYC_BEGIN() do {} while (0)
+#define QL_CYC_END(i) do {} while (0)
+#define QL_CYC_ADD(i, v) do {} while (0)
+#define QL_CYC_FLUSH() do {} while (0)
+#endif
+
+// Ablation switches for timing experiments (sp.ablate; the results are garbage when any is set):
+// 1 no weight copies, unpacking or MMAs, 2 X operand not loaded or converted, 4 1/rms not awaited,
+// 8 split tiles not exchanged, 16 rows published without the fence, 32 no accumulator exchange,
+// 64 no row epilogue (publish only), 256 watcher without its acquire fence
 struct WaitCtx {
   volatile int* s_abort;
   int* status;
@@ -120,6 +159,7 @@ __device__ __forceinline__ void wait_shared_gt(volatile int* p, int seen, const 
   const uint64_t t0 = globaltimer_ns();
   uint32_t spins = 0;
   while (*p <= seen) {
+    __nanosleep(32);                                     // leave the issue slots to the warps that work
     if ((++spins & 63u) == 0) {
       if (*w.s_abort) return;
       if (globaltimer_ns() - t0 > w.budget) { wait_fail(w, site); return; }
@@ -144,6 +184,133 @@ __device__ __forceinline__ OpHead load_head(const MegaOp* op) {
 template <typename T>
 __device__ __forceinline__ T* ldg_ptr(T* const* p) {
   return reinterpret_cast<T*>(__ldg(reinterpret_cast<const unsigned long long*>(p)));
+}
+
+// X duty of one operation (all 512 unpack threads, no barrier among them): waits until the watcher
+// has seen the previous operation complete, then builds the CTA's share of the X operand in shared
+// memory - 16-byte units (8 consecutive k of one row) in the K-major core-matrix layout the MMA
+// reads, slot k holding the group of the CTA's chunk number k.  `d` is the operation's descriptor
+// in shared memory.  All loads of a thread are issued before the first is used.
+template <int G>
+__device__ __forceinline__ void build_x(const StackParams& sp, const MegaOp& d, int j, uint8_t* xbuf, const float* s_inv,
+                                     volatile int* s_dep, volatile int* s_invrdy, uint64_t* x_full, const WaitCtx& wc,
+                                     uint32_t start, uint32_t my_chunks, uint32_t Gn) {
+  constexpr uint32_t XSLOT = st_xslot_bytes(G);
+  constexpr uint32_t UPR = G / 8;                       // 16-byte units per row of one group
+  constexpr uint32_t UPG = (uint32_t)MP * UPR;          // per group
+  const int tid = threadIdx.x, lane = tid & 31;
+  const uint32_t cta = blockIdx.x;
+  (void)cta;
+  const uint32_t n_x = min(my_chunks, Gn);
+  const uint32_t g_first = start % Gn;
+  const uint32_t n_units = n_x * UPG;
+  const int prologue = d.prologue;
+  const int ld_in = d.ld_in;
+  const uint16_t* in0 = d.in0;
+  // unit idx: slot k = idx / UPG, row m = (idx / UPR) % MP, k-unit ku = idx % UPR: lanes run along K
+  auto unit_addr = [&](uint32_t idx) -> uint8_t* {
+    const uint32_t k = idx / UPG, r = idx % UPG, m = r / UPR, ku = r % UPR;
+    return xbuf + (size_t)k * XSLOT + ku * kXLbo + (m >> 3) * 128u + (m & 7u) * 16u;
+  };
+  auto unit_col = [&](uint32_t idx) -> size_t {          // first column (k index) of the unit in the source row
+    const uint32_t k = idx / UPG, ku = idx % UPR;
+    uint32_t Gi = g_first + k;
+    if (Gi >= Gn) Gi -= Gn;
+    return (size_t)Gi * G + ku * 8;
+  };
+  auto unit_row = [&](uint32_t idx) -> uint32_t { return (idx % UPG) / UPR; };
+  wait_shared_gt(s_dep, j, wc, 8);
+  __threadfence_block();
+  QL_STAMP(2);
+  if (sp.ablate & 2) {
+    if (prologue != 0 && !(sp.ablate & 4)) { wait_shared_gt(s_invrdy, j, wc, 9); }
+  } else if (prologue == 0) {
+    for (uint32_t idx = tid; idx < n_units; idx += kUnpackThreads) {
+      const uint32_t m = unit_row(idx);
+      const bool live = (int)m < sp.M;
+      cp_async16(unit_addr(idx), live ? (in0 + (size_t)m * ld_in + unit_col(idx)) : in0, live ? 16u : 0u);
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");
+  } else {
+    // X = bf16(v * 1/rms): v is the producer's bf16 output (prologue 1) or the fp32 product
+    // silu(gate) * up it left in the workspace (prologue 2); 1/rms arrives from the watcher meanwhile.
+    uint16_t* xout = d.xout;
+    const int ld_xout = d.ld_xout;
+    auto emit = [&](uint32_t idx, uint4 o) {
+      const uint32_t m = unit_row(idx);
+      // the CTA that owns (tile 0, group Gi) writes the normalised X out for the record
+      if (xout != nullptr && (int)m < sp.M && start + idx / UPG < Gn)
+        *reinterpret_cast<uint4*>(xout + (size_t)m * ld_xout + unit_col(idx)) = o;
+      *reinterpret_cast<uint4*>(unit_addr(idx)) = o;
+    };
+    bool have_inv = false;
+    auto need_inv = [&]() {
+      if (!have_inv && !(sp.ablate & 4)) {
+        wait_shared_gt(s_invrdy, j, wc, 9);
+        __threadfence_block();
+        have_inv = true;
+      }
+    };
+    if (prologue == 1) {
+      constexpr int XB = 10;                             // 10 units per thread cover 20 groups
+      for (uint32_t base = tid; base < n_units; base += kUnpackThreads * XB) {
+        uint4 ra[XB];
+#pragma unroll
+        for (int q = 0; q < XB; ++q) {
+          const uint32_t idx = base + q * kUnpackThreads;
+          ra[q] = make_uint4(0u, 0u, 0u, 0u);
+          if (idx < n_units && (int)unit_row(idx) < sp.M)
+            ra[q] = __ldcg(reinterpret_cast<const uint4*>(in0 + (size_t)unit_row(idx) * ld_in + unit_col(idx)));
+        }
+        need_inv();
+#pragma unroll
+        for (int q = 0; q < XB; ++q) {
+          const uint32_t idx = base + q * kUnpackThreads;
+          if (idx >= n_units) continue;
+          const float inv = (int)unit_row(idx) < sp.M ? s_inv[unit_row(idx)] : 0.f;
+          uint4 o;
+          o.x = pack_bf16x2_rn(bf16lo_to_f32(ra[q].x) * inv, bf16hi_to_f32(ra[q].x) * inv);
+          o.y = pack_bf16x2_rn(bf16lo_to_f32(ra[q].y) * inv, bf16hi_to_f32(ra[q].y) * inv);
+          o.z = pack_bf16x2_rn(bf16lo_to_f32(ra[q].z) * inv, bf16hi_to_f32(ra[q].z) * inv);
+          o.w = pack_bf16x2_rn(bf16lo_to_f32(ra[q].w) * inv, bf16hi_to_f32(ra[q].w) * inv);
+          emit(idx, o);
+        }
+      }
+    } else {
+      constexpr int XB = 6;                              // 6 units per thread cover 12 groups
+      const float* act = sp.ws.act;
+      const int K = d.K;
+      for (uint32_t base = tid; base < n_units; base += kUnpackThreads * XB) {
+        uint4 ra[XB], rb[XB];
+#pragma unroll
+        for (int q = 0; q < XB; ++q) {
+          const uint32_t idx = base + q * kUnpackThreads;
+          ra[q] = make_uint4(0u, 0u, 0u, 0u); rb[q] = ra[q];
+          if (idx < n_units && (int)unit_row(idx) < sp.M) {
+            const uint4* p = reinterpret_cast<const uint4*>(act + (size_t)unit_row(idx) * K + unit_col(idx));
+            ra[q] = __ldcg(p);
+            rb[q] = __ldcg(p + 1);
+          }
+        }
+        need_inv();
+#pragma unroll
+        for (int q = 0; q < XB; ++q) {
+          const uint32_t idx = base + q * kUnpackThreads;
+          if (idx >= n_units) continue;
+          const float inv = (int)unit_row(idx) < sp.M ? s_inv[unit_row(idx)] : 0.f;
+          uint4 o;
+          o.x = pack_bf16x2_rn(__uint_as_float(ra[q].x) * inv, __uint_as_float(ra[q].y) * inv);
+          o.y = pack_bf16x2_rn(__uint_as_float(ra[q].z) * inv, __uint_as_float(ra[q].w) * inv);
+          o.z = pack_bf16x2_rn(__uint_as_float(rb[q].x) * inv, __uint_as_float(rb[q].y) * inv);
+          o.w = pack_bf16x2_rn(__uint_as_float(rb[q].z) * inv, __uint_as_float(rb[q].w) * inv);
+          emit(idx, o);
+        }
+      }
+    }
+  }
+  fence_proxy_async();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(x_full);
 }
 
 template <int G>
@@ -174,6 +341,9 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_flag + 9);
   volatile int* s_dep = s_flag + 10;                    // operations whose predecessor is known to be complete
   volatile int* s_invrdy = s_flag + 11;                 // operations whose 1/rms values are in s_inv
+  volatile int* s_descrdy = s_flag + 12;                // operations whose descriptor is in s_desc
+  volatile int* s_prog = s_flag + 16;                   // [16] operations each unpack warp has left behind
+  MegaOp* s_desc = reinterpret_cast<MegaOp*>(s_flag + 32);   // [2] descriptors of operations j (slot j & 1), filled by the watcher
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const MegaOp* __restrict__ ops = sp.ops;
@@ -194,6 +364,8 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
     *s_abort = 0;
     *s_dep = 0;
     *s_invrdy = 0;
+    *s_descrdy = 0;
+    for (int i = 0; i < 16; ++i) s_prog[i] = 0;
     fence_mbar_init();
   }
   if (warp == kWarpIssuer0) {
@@ -216,6 +388,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
         uint32_t start, end;
         op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
         if (start >= end) continue;
+        if (sp.ablate & 1) continue;
         const uint8_t* p0 = ldg_ptr(&ops[j].packed0);
         const uint8_t* p1 = ldg_ptr(&ops[j].packed1);
         const int nmat = (h.flags & kOpDual) ? 2 : 1;
@@ -241,17 +414,42 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
       }
     }
   } else if (warp == kWarpWatcher) {
-    // ------------------------------------------------------------------ watcher: dependencies and row scales
+    // ------------------------------------------------------------------ watcher: descriptors, dependencies, row scales
     for (int j = 0; j < sp.n_ops; ++j) {
+      // the unpack warps read the descriptor of operation j from shared memory (slot j & 1); the
+      // slot is free once every unpack warp has left operation j-2 behind
+      if (j >= 2) {
+        const uint64_t t0 = globaltimer_ns();
+        for (;;) {
+          int p = lane < 16 ? s_prog[lane] : 0x7fffffff;
+#pragma unroll
+          for (int off = 8; off >= 1; off >>= 1) p = min(p, __shfl_xor_sync(0xffffffffu, p, off));
+          p = __shfl_sync(0xffffffffu, p, 0);
+          if (p >= j - 1 || *s_abort) break;
+          if (globaltimer_ns() - t0 > wc.budget) { if (lane == 0) wait_fail(wc, 12); break; }
+          __nanosleep(64);
+        }
+      }
+      if (lane < 8) reinterpret_cast<uint4*>(&s_desc[j & 1])[lane] = __ldg(reinterpret_cast<const uint4*>(ops + j) + lane);
+      __syncwarp();
+      if (lane == 0) {
+        __threadfence_block();
+        *s_descrdy = j + 1;
+      }
       const OpHead h = load_head(ops + j);
-      if (j > 0 && (h.flags & kOpWait)) {
-        if (lane == 0) {
-          const int need = __ldg(&ops[j - 1].n_tiles);
-          wait_global<true>(&sp.ws.op_done[j - 1], need, wc, 7);
+      // an operation waits for the one before it (it consumes its output), or only for the one two
+      // back (independent operations: the partial-tile slots and flags alternate between two sets)
+      const int dep = (h.flags & kOpWait) ? j - 1 : ((h.flags & kOpWait2) ? j - 2 : -1);
+      if (dep >= 0) {
+        // every tile is published row by row; lane r polls the counter of row r (one line per counter)
+        if (lane < 16) {
+          const int need = __ldg(&ops[dep].n_tiles);
+          wait_global<true>(&sp.ws.op_done[((size_t)dep * 16 + lane) * kOpDoneStride], need, wc, 7);
         }
         __syncwarp();
-        fence_gpu();                                     // acquire: everything the finishers published
+        if (!(sp.ablate & 256)) fence_gpu();             // acquire: everything the finishers published
       }
+      QL_STAMP_W(7);
       if (lane == 0) {
         __threadfence_block();
         *s_dep = j + 1;
@@ -266,12 +464,12 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
         const float* ssq = sp.ws.ssq + (size_t)((j - 1) & 1) * sp.ws.n_tiles * 16;
         const int row = lane & 15, half = lane >> 4;
         float sum = 0.f;
-        for (int t0 = half; t0 < src_tiles; t0 += 16) {
-          float v[8];
+        for (int t0 = half; t0 < src_tiles; t0 += 80) {   // 40 loads in flight per lane: one round trip up to 80 tiles
+          float v[40];
 #pragma unroll
-          for (int q = 0; q < 8; ++q) v[q] = (t0 + 2 * q < src_tiles) ? __ldcg(&ssq[(size_t)(t0 + 2 * q) * 16 + row]) : 0.f;
+          for (int q = 0; q < 40; ++q) v[q] = (t0 + 2 * q < src_tiles) ? __ldcg(&ssq[(size_t)(t0 + 2 * q) * 16 + row]) : 0.f;
 #pragma unroll
-          for (int q = 0; q < 8; ++q) sum += v[q];
+          for (int q = 0; q < 40; ++q) sum += v[q];
         }
         const float other = __shfl_xor_sync(0xffffffffu, sum, 16);
         const float tot = half == 0 ? sum + other : other + sum;
@@ -284,11 +482,12 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
       }
       if (*s_abort) break;
     }
+    if (lane == 0 && *s_abort) { *s_descrdy = 0x7ffffff0; *s_dep = 0x7ffffff0; *s_invrdy = 0x7ffffff0; }
   } else if (warp >= kWarpIssuer0) {
     // ------------------------------------------------------------------ MMA issue for unpack group w
     if (lane == 0) {
       constexpr uint32_t idesc = tc_idesc_bf16_m128(MP);
-      const uint32_t w = warp - kWarpIssuer0;
+      const uint32_t w = warp - kWarpIssuer0;             // unpack group served
       const uint64_t desc0 = tc_smem_desc_kmajor(smem_u32(xbuf), kXLbo, 128u);
       constexpr uint32_t KSTEP = (2u * kXLbo) >> 4;     // one MMA contracts 16 rows of K = two core matrices
       constexpr uint32_t SLOT = XSLOT >> 4;
@@ -296,6 +495,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
       uint32_t k = 0;                                  // chunks this group has handed over so far
       uint32_t hs = 0;                                 // half-chunks
       uint32_t xops = 0;                               // operations this CTA took part in so far
+      QL_CYC_DECL;
       for (int j = 0; j < sp.n_ops; ++j) {
         const OpHead h = load_head(ops + j);
         uint32_t start, end;
@@ -305,6 +505,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
         const uint32_t Gn = (uint32_t)h.n_groups;
         const uint32_t n_sub = (end - start) * (dual ? 2u : 1u);
         ++xops;
+        if (sp.ablate & 1) continue;
         bool first = true;
         for (uint32_t e = w; e < n_sub; e += NWG, ++k) {
           uint32_t xk = dual ? (e >> 1) : e;           // X slot = chunk number within the CTA, modulo the group count
@@ -314,11 +515,14 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh, ++hs) {
             const uint32_t slot = hs % AH;
+            QL_CYC_BEGIN();
             st_mbar_wait(&a_full[w * AH + slot], (hs / AH) & 1, wc, 3);
+            QL_CYC_END(0);
             if (first) {
               st_mbar_wait(x_full, (xops - 1) & 1, wc, 2);   // X of this operation is in shared memory
               first = false;
             }
+            QL_CYC_END(1);
             tc_fence_after_sync();
 #pragma unroll
             for (int jj = 0; jj < NK / 2; ++jj) {
@@ -326,10 +530,13 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
               tc_mma_ts_f16(d_tmem, a_base + slot * AHC + 8 * jj, xdesc + (uint64_t)(jk * KSTEP), idesc, jk > 0 ? 1u : 0u);
             }
             tc_commit(&a_empty[w * AH + slot]);
+            QL_CYC_END(2);
+            QL_CYC_ADD(3, 1);
           }
           tc_commit(&d_full[2 * w + (k & 1)]);
         }
       }
+      QL_CYC_FLUSH_I();
     }
   } else {
     // ------------------------------------------------------------------ unpack groups
@@ -339,132 +546,103 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
     const uint32_t tlane = tmem + ((uint32_t)(wq * 32) << 16);
     const uint32_t a_addr = tlane + w * AH * AHC;
     const uint32_t d_addr = tlane + D_COL0 + 2 * w * MP;
-    uint64_t* my_slot = reinterpret_cast<uint64_t*>(sp.ws.slots) + (size_t)cta * kSlotWords;
+    constexpr uint32_t kSetCtas = kMaxCtas / 2;          // partial-tile slots and row flags: two sets of 160
     uint32_t stg = 0, sph = 0;                          // ring stage / phase of the next sub-chunk (any group's)
     uint32_t kloc = 0;                                  // chunks this group has handed to the tensor core
     uint32_t hs = 0;                                    // half-chunks this group has stored
     float acc[MP];
+    QL_CYC_DECL;
 
     auto drain = [&](uint32_t kq, float s_q) {
       const uint32_t b = kq & 1;
+      QL_CYC_BEGIN();
       st_mbar_wait(&d_full[2 * w + b], (kq >> 1) & 1, wc, 4);
+      QL_CYC_END(4);
       tc_fence_after_sync();
       float d[16];
       tmem_ld16(d_addr + b * MP, d);
       tmem_wait_ld();
 #pragma unroll
       for (int m = 0; m < 16; ++m) acc[m] = fmaf(s_q, d[m], acc[m]);
+      QL_CYC_END(5);
     };
 
     for (int j = 0; j < sp.n_ops; ++j) {
-      const OpHead h = load_head(ops + j);
+      // the watcher has put the descriptor into shared memory (normally long before)
+      if (lane == 0) wait_shared_gt(s_descrdy, j, wc, 13);
+      __syncwarp();
+      __threadfence_block();
+      const MegaOp& dsc = s_desc[j & 1];
+      OpHead h;
+      h.nc = dsc.nc; h.cq = dsc.cq; h.cr = dsc.cr; h.cat_base = dsc.cat_base;
+      h.total_chunks = dsc.total_chunks; h.n_groups = dsc.n_groups; h.n_tiles = dsc.n_tiles; h.flags = dsc.flags;
       uint32_t start, end;
       op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
-      if (start >= end) continue;
-      const MegaOp* op = ops + j;
+      if (start >= end) {
+        __syncwarp();
+        if (lane == 0) s_prog[warp] = j + 1;
+        continue;
+      }
       const bool dual = (h.flags & kOpDual) != 0;
       const uint32_t Gn = (uint32_t)h.n_groups;
       const uint32_t my_chunks = end - start;
       const uint32_t tag = (sp.epoch << 9) | (uint32_t)(j + 1);
-      bool x_done = false;
-      uint32_t pre = 0;                                 // half-chunks of this operation stored before its X exists
+      const uint32_t n_sub_total = my_chunks * (dual ? 2u : 1u);
+      QL_STAMP(0);
 
-      // -------- X duty (all 512 threads): wait for the previous operation, build the X operand --------
-      auto x_duty = [&]() {
-        constexpr uint32_t UPG = (uint32_t)MP * (G / 8);   // 16-byte units per group
-        const uint32_t n_x = min(my_chunks, Gn);
-        const uint32_t g_first = start % Gn;
-        const uint32_t n_units = n_x * UPG;
-        const int prologue = __ldg(&op->prologue);
-        const int ld_in = __ldg(&op->ld_in);
-        const uint16_t* in0 = ldg_ptr(&op->in0);
-        // unit idx: slot k = idx / UPG, row m = (idx / (G/8)) % MP, k-unit ku = idx % (G/8): lanes run along K
-        auto unit_addr = [&](uint32_t k, uint32_t m, uint32_t ku) -> uint8_t* {
-          return xbuf + (size_t)k * XSLOT + ku * kXLbo + (m >> 3) * 128u + (m & 7u) * 16u;
-        };
-        wait_shared_gt(s_dep, j, wc, 8);
-        __threadfence_block();
-        if (prologue == 0) {
-          for (uint32_t idx = tid; idx < n_units; idx += kUnpackThreads) {
-            const uint32_t k = idx / UPG, r = idx % UPG;
-            const uint32_t m = r / (G / 8), ku = r % (G / 8);
-            uint32_t Gi = g_first + k;
-            if (Gi >= Gn) Gi -= Gn;
-            const bool live = (int)m < sp.M;
-            cp_async16(unit_addr(k, m, ku), live ? (in0 + (size_t)m * ld_in + (size_t)Gi * G + ku * 8) : in0, live ? 16u : 0u);
+      // Expands one packed chunk (ring stage s) into two half-chunk A buffers of this group and
+      // hands them to the issuer; returns the column's scale.
+      auto unpack_subchunk = [&](uint32_t s, uint32_t ph) -> float {
+        const uint8_t* st = ring + (size_t)s * STAGE;
+        QL_CYC_BEGIN();
+        st_mbar_wait(&full[s], ph, wc, 5);
+        QL_CYC_END(0);
+        QL_CYC_ADD(6, 1);
+        const float sc = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(st + 64 * G)[n] << 16);
+        const uint32_t z = (reinterpret_cast<const uint32_t*>(st + 64 * G + 256)[n >> 3] >> (4 * (n & 7))) & 0xFu;
+        const uint32_t zb = 0x43004300u | z | (z << 16);
+        const uint4* wst = reinterpret_cast<const uint4*>(st);
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh, ++hs) {
+          const uint32_t slot = hs % AH;
+          if (hs >= AH) {
+            st_mbar_wait(&a_empty[w * AH + slot], ((hs / AH) - 1) & 1, wc, 6);
+            tc_fence_after_sync();
           }
-          asm volatile("cp.async.wait_all;" ::: "memory");
-        } else {
-          // X = bf16(v * 1/rms): v is the producer's bf16 output (prologue 1) or the fp32 product
-          // silu(gate) * up it left in the workspace (prologue 2).  The loads of a batch are all
-          // issued before any is used; 1/rms arrives from the watcher meanwhile.
-          constexpr int XB = 4;
-          const bool from_act = (prologue == 2);
-          const float* act = sp.ws.act;
-          const int K = __ldg(&op->K);
-          uint16_t* xout = ldg_ptr(&op->xout);
-          const int ld_xout = __ldg(&op->ld_xout);
-          bool have_inv = false;
-          for (uint32_t base = tid; base < n_units; base += kUnpackThreads * XB) {
-            uint4 ra[XB], rb[XB];
-            uint32_t kk[XB], mm[XB], uu[XB], gg[XB];
+          QL_CYC_END(1);
 #pragma unroll
-            for (int q = 0; q < XB; ++q) {
-              const uint32_t idx = base + q * kUnpackThreads;
-              const bool in_range = idx < n_units;
-              const uint32_t k = in_range ? idx / UPG : 0, r = idx % UPG;
-              const uint32_t m = r / (G / 8), ku = r % (G / 8);
-              uint32_t Gi = g_first + k;
-              if (Gi >= Gn) Gi -= Gn;
-              kk[q] = k; mm[q] = m; uu[q] = ku; gg[q] = Gi;
-              ra[q] = make_uint4(0u, 0u, 0u, 0u); rb[q] = ra[q];
-              if (in_range && (int)m < sp.M) {
-                const size_t col0 = (size_t)Gi * G + ku * 8;
-                if (from_act) {
-                  const uint4* p = reinterpret_cast<const uint4*>(act + (size_t)m * K + col0);
-                  ra[q] = __ldcg(p);
-                  rb[q] = __ldcg(p + 1);
-                } else {
-                  ra[q] = __ldcg(reinterpret_cast<const uint4*>(in0 + (size_t)m * ld_in + col0));
-                }
-              }
-            }
-            if (!have_inv) {
-              wait_shared_gt(s_invrdy, j, wc, 9);
-              __threadfence_block();
-              have_inv = true;
-            }
-#pragma unroll
-            for (int q = 0; q < XB; ++q) {
-              const uint32_t idx = base + q * kUnpackThreads;
-              if (idx >= n_units) continue;
-              uint4 o = make_uint4(0u, 0u, 0u, 0u);
-              if ((int)mm[q] < sp.M) {
-                const float inv = s_inv[mm[q]];
-                if (!from_act) {
-                  o.x = pack_bf16x2_rn(bf16lo_to_f32(ra[q].x) * inv, bf16hi_to_f32(ra[q].x) * inv);
-                  o.y = pack_bf16x2_rn(bf16lo_to_f32(ra[q].y) * inv, bf16hi_to_f32(ra[q].y) * inv);
-                  o.z = pack_bf16x2_rn(bf16lo_to_f32(ra[q].z) * inv, bf16hi_to_f32(ra[q].z) * inv);
-                  o.w = pack_bf16x2_rn(bf16lo_to_f32(ra[q].w) * inv, bf16hi_to_f32(ra[q].w) * inv);
-                } else {
-                  o.x = pack_bf16x2_rn(__uint_as_float(ra[q].x) * inv, __uint_as_float(ra[q].y) * inv);
-                  o.y = pack_bf16x2_rn(__uint_as_float(ra[q].z) * inv, __uint_as_float(ra[q].w) * inv);
-                  o.z = pack_bf16x2_rn(__uint_as_float(rb[q].x) * inv, __uint_as_float(rb[q].y) * inv);
-                  o.w = pack_bf16x2_rn(__uint_as_float(rb[q].z) * inv, __uint_as_float(rb[q].w) * inv);
-                }
-                // the CTA that owns (tile 0, group Gi) writes the normalised X out for the record
-                if (xout != nullptr && start + kk[q] < Gn)
-                  *reinterpret_cast<uint4*>(xout + (size_t)mm[q] * ld_xout + (size_t)gg[q] * G + uu[q] * 8) = o;
-              }
-              *reinterpret_cast<uint4*>(unit_addr(kk[q], mm[q], uu[q])) = o;
-            }
+          for (int cc = 0; cc < NC / 2; ++cc) {
+            uint32_t v[16];
+            unpack_codes32(wst[(hh * (NC / 2) + cc) * kTileN + n], zb, v);
+            tmem_st16(a_addr + slot * AHC + 16 * cc, v);
+          }
+          QL_CYC_END(2);
+          tmem_wait_st();
+          QL_CYC_END(3);
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(&a_full[w * AH + slot]);
+            if (hh == 1) mbar_arrive(&empty[s]);
           }
         }
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(x_full);
-        x_done = true;
+        return sc;
       };
+
+      // -------- the group's first chunk of the operation is unpacked BEFORE its X exists (the A
+      //          operand depends on weights only; the issuer holds the MMAs back) --------
+      float pre_sc = 0.f;
+      uint32_t pre_e = 0xffffffffu;                     // sub-chunk of this group that is already unpacked
+      if ((uint32_t)w < n_sub_total && !(sp.ablate & 1)) {
+        uint32_t s = stg + (uint32_t)w, ph = sph;
+        if (s >= (uint32_t)NS) { s -= (uint32_t)NS; ph ^= 1; }
+        pre_sc = unpack_subchunk(s, ph);
+        pre_e = (uint32_t)w;
+      }
+      QL_STAMP(1);
+      // -------- X duty (all 512 threads): wait for the previous operation, build the X operand --------
+      build_x<G>(sp, dsc, j, xbuf, s_inv, s_dep, s_invrdy, x_full, wc, start, my_chunks, Gn);
+      QL_STAMP(3);
 
       // -------- chunks of this operation --------
       uint32_t pos = start, e = 0;                      // e: sub-chunk counter of the operation (this CTA)
@@ -483,53 +661,40 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
           const uint32_t my_stage = stg, my_phase = sph;
           if (++stg == (uint32_t)NS) { stg = 0; sph ^= 1; }
           if ((int)(e % NWG) != w) continue;
-          const uint8_t* st = ring + (size_t)my_stage * STAGE;
-          st_mbar_wait(&full[my_stage], my_phase, wc, 5);
-          const float sc = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(st + 64 * G)[n] << 16);
-          const uint32_t z = (reinterpret_cast<const uint32_t*>(st + 64 * G + 256)[n >> 3] >> (4 * (n & 7))) & 0xFu;
-          const uint32_t zb = 0x43004300u | z | (z << 16);
-          const uint4* wst = reinterpret_cast<const uint4*>(st);
-          if (n_pend == 2) { drain(kloc - 2, s_p2); n_pend = 1; }
-#pragma unroll
-          for (int hh = 0; hh < 2; ++hh, ++hs) {
-            // the A buffers hold AH half-chunks: whatever fits is unpacked before X exists, then
-            // the group turns to the X operand, whose MMAs free the buffers again
-            if (!x_done && pre == AH) x_duty();
-            ++pre;
-            const uint32_t slot = hs % AH;
-            if (hs >= AH) {
-              st_mbar_wait(&a_empty[w * AH + slot], ((hs / AH) - 1) & 1, wc, 6);
-              tc_fence_after_sync();
-            }
-#pragma unroll
-            for (int cc = 0; cc < NC / 2; ++cc) {
-              uint32_t v[16];
-              unpack_codes32(wst[(hh * (NC / 2) + cc) * kTileN + n], zb, v);
-              tmem_st16(a_addr + slot * AHC + 16 * cc, v);
-            }
-            tmem_wait_st();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) {
-              mbar_arrive(&a_full[w * AH + slot]);
-              if (hh == 1) mbar_arrive(&empty[my_stage]);
-            }
+          float sc;
+          if (sp.ablate & 1) {
+            sc = 0.f;
+          } else if (e == pre_e) {
+            sc = pre_sc;                                 // unpacked ahead (before X duty, or before the previous tile end)
+          } else {
+            if (n_pend == 2) { drain(kloc - 2, s_p2); n_pend = 1; }
+            sc = unpack_subchunk(my_stage, my_phase);
           }
+          if (sp.ablate & 1) n_pend = 0;
           s_p2 = s_p1;
           s_p1 = sc;
           ++n_pend;
           ++kloc;
         }
-        if (!x_done) x_duty();                           // fewer than AH half-chunks before the segment's end
-        if (n_pend == 2) drain(kloc - 2, s_p2);
-        if (n_pend >= 1) drain(kloc - 1, s_p1);
+        if (!(sp.ablate & 1)) {
+          if (n_pend == 2) drain(kloc - 2, s_p2);
+          if (n_pend >= 1) drain(kloc - 1, s_p1);
+        }
         tc_fence_before_sync();
+        if (pos == start) QL_STAMP(4);
+        if (pos + nch == end) QL_STAMP(8);
 
-        // ---- end of a tile segment: the four groups' accumulators meet in shared memory; from here
-        //      on warp r owns row r of the tile and lane l its columns 4l..4l+3 ----
+        // ---- end of a tile segment: the four groups' accumulators meet in shared memory.  From the
+        //      second barrier on, every warp works alone: warp r owns row r of the tile (lane l its
+        //      columns 4l..4l+3), exchanges row r of split tiles, stores it and publishes it. ----
+        if (!(sp.ablate & 32)) {
+        named_bar_sync(1, kUnpackThreads);               // every warp is done reading the previous segment's sums
 #pragma unroll
         for (int m = 0; m < MP; ++m) red[(w * MP + m) * kTileN + n] = acc[m];
         named_bar_sync(1, kUnpackThreads);
+        }
+        if (pos == start) QL_STAMP(5);
+        if (pos + nch == end) QL_STAMP(9);
         const int rw = warp;
         float f0[4], f1[4] = {0.f, 0.f, 0.f, 0.f};
         {
@@ -545,76 +710,67 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
           }
         }
         const bool whole = (g0 == 0 && nch == Gn);
-        const bool finish = (g0 == 0);                   // my run contains the tile's first chunk
+        bool finish = (g0 == 0);                         // my run contains the tile's first chunk
+        if ((sp.ablate & 8) && !whole && !finish) { pos += nch; continue; }
         pos += nch;
         const int nmat = dual ? 2 : 1;
+        int* row_flag = sp.ws.tile_cnt + (j & 1) * (16 * kSetCtas) + rw;   // flag of (CTA i, row r) at [16 i + r] of the set j & 1
+        float* set_slots = sp.ws.slots + (size_t)(j & 1) * kSetCtas * kSlotWords;
+        float* my_slot = set_slots + (size_t)cta * kSlotWords;
 
         if (!whole && !finish) {
-          // ---- contributor: (value, tag) pairs, then the flag; no fence in between - the owner
-          //      checks every tag.  (A run that does not begin its tile meets it in its first
-          //      segment, so one slot per CTA is enough.) ----
+          // ---- contributor: row r of its partial tile, one fence over the warp's stores, then the
+          //      row's flag.  (A run that does not begin its tile meets it in its first segment, so
+          //      one slot per CTA is enough.) ----
           for (int mt = 0; mt < nmat; ++mt) {
             const float* f = mt ? f1 : f0;
-            uint64_t* dst = my_slot + (size_t)(mt * MP + rw) * kTileN + 4 * lane;
-            st_pairs(dst, tagged(f[0], tag), tagged(f[1], tag));
-            st_pairs(dst + 2, tagged(f[2], tag), tagged(f[3], tag));
+            __stcg(reinterpret_cast<float4*>(my_slot + (size_t)(mt * MP + rw) * kTileN + 4 * lane), make_float4(f[0], f[1], f[2], f[3]));
           }
-          named_bar_sync(1, kUnpackThreads);             // red is free; everybody's pairs are on their way
-          if (tid == 0) st_relaxed(&sp.ws.tile_cnt[cta], (int)tag);
+          __syncwarp();
+          if (lane == 0) {
+            fence_gpu();
+            st_relaxed(&row_flag[16 * cta], (int)tag);
+          }
+          if (pos - nch == start) QL_STAMP(6);
+          if (pos == end) QL_STAMP(14);
           continue;
         }
-        if (!whole) {
+        if (!whole && !(sp.ablate & 8)) {
           // ---- owner of a split tile: its own partial stays in registers; the others' are added in
-          //      CTA order once their flags are up ----
-          if (tid == 0) s_flag[1] = (int)run_chunk_owner(h.nc, h.cq, h.cr, h.cat_base + T * Gn + Gn - 1);
-          named_bar_sync(1, kUnpackThreads);
-          const uint32_t last = (uint32_t)s_flag[1];
-          for (uint32_t i = cta + 1 + tid; i <= last; i += kUnpackThreads)
-            wait_global<false>(&sp.ws.tile_cnt[i], (int)tag, wc, 10);
-          named_bar_sync(1, kUnpackThreads);
-          const uint64_t* slots64 = reinterpret_cast<const uint64_t*>(sp.ws.slots);
+          //      CTA order once their flags for this row are up (lane q polls contributor q) ----
+          const uint32_t last = run_chunk_owner(h.nc, h.cq, h.cr, h.cat_base + T * Gn + Gn - 1);
+          for (uint32_t i = cta + 1 + lane; i <= last; i += 32) wait_global<false>(&row_flag[16 * i], (int)tag, wc, 10);
+          __syncwarp();
+          fence_gpu();                                     // acquire: the contributors' rows
+          if (pos == end) QL_STAMP(10);
           for (int mt = 0; mt < nmat; ++mt) {
             float* f = mt ? f1 : f0;
-            for (uint32_t i0 = cta + 1; i0 <= last; i0 += 2) {
-              uint64_t v[2][4];
+            for (uint32_t i0 = cta + 1; i0 <= last; i0 += 8) {
+              float4 v[8];
 #pragma unroll
-              for (int q = 0; q < 2; ++q) {
+              for (int q = 0; q < 8; ++q) {
                 const uint32_t i = min(i0 + q, last);
-                const uint64_t* src = slots64 + (size_t)i * kSlotWords + (size_t)(mt * MP + rw) * kTileN + 4 * lane;
-                ld_pairs(src, v[q][0], v[q][1]);
-                ld_pairs(src + 2, v[q][2], v[q][3]);
+                v[q] = __ldcg(reinterpret_cast<const float4*>(set_slots + (size_t)i * kSlotWords + (size_t)(mt * MP + rw) * kTileN + 4 * lane));
               }
 #pragma unroll
-              for (int q = 0; q < 2; ++q) {
+              for (int q = 0; q < 8; ++q) {
                 if (i0 + q > last) continue;
-                bool ok = (uint32_t)(v[q][0] >> 32) == tag && (uint32_t)(v[q][1] >> 32) == tag &&
-                          (uint32_t)(v[q][2] >> 32) == tag && (uint32_t)(v[q][3] >> 32) == tag;
-                if (!ok && !*s_abort) {
-                  // the flag overtook some of the pairs: reload until every tag matches (bounded)
-                  const uint64_t* src = slots64 + (size_t)(i0 + q) * kSlotWords + (size_t)(mt * MP + rw) * kTileN + 4 * lane;
-                  const uint64_t t0 = globaltimer_ns();
-                  while (!ok) {
-                    ld_pairs(src, v[q][0], v[q][1]);
-                    ld_pairs(src + 2, v[q][2], v[q][3]);
-                    ok = (uint32_t)(v[q][0] >> 32) == tag && (uint32_t)(v[q][1] >> 32) == tag &&
-                         (uint32_t)(v[q][2] >> 32) == tag && (uint32_t)(v[q][3] >> 32) == tag;
-                    if (!ok && (*s_abort || globaltimer_ns() - t0 > wc.budget)) { wait_fail(wc, 11); break; }
-                  }
-                }
-#pragma unroll
-                for (int r = 0; r < 4; ++r) f[r] += __uint_as_float((uint32_t)v[q][r]);
+                f[0] += v[q].x; f[1] += v[q].y; f[2] += v[q].z; f[3] += v[q].w;
               }
             }
           }
         }
 
-        // ---- tile epilogue: bf16 stores, sums of squares for the next operation, arg-max ----
-        {
-          uint16_t* out0 = ldg_ptr(&op->out0);
-          uint16_t* out1 = ldg_ptr(&op->out1);
-          int32_t* argmax_out = ldg_ptr(&op->argmax_out);
-          const int emit_ssq = __ldg(&op->emit_ssq);
-          const int ld_out = __ldg(&op->ld_out);
+        if (pos == end) QL_STAMP(11);
+        // ---- row epilogue: bf16 stores, sum of squares for the next operation, arg-max ----
+        if (sp.ablate & 64) {
+          __syncwarp();
+          if (lane == 0) red_relaxed_add(&sp.ws.op_done[((size_t)j * 16 + rw) * kOpDoneStride], 1);
+        } else {
+          uint16_t* out0 = dsc.out0;
+          int32_t* argmax_out = dsc.argmax_out;
+          const int emit_ssq = dsc.emit_ssq;
+          const int ld_out = dsc.ld_out;
           const int col = (int)T * kTileN + 4 * lane;
           const bool live = rw < sp.M;
           float a[4];
@@ -627,12 +783,12 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
             uint2 y1;
             y1.x = pack_bf16x2_rn(f1[0], f1[1]);
             y1.y = pack_bf16x2_rn(f1[2], f1[3]);
-            if (live) *reinterpret_cast<uint2*>(out1 + (size_t)rw * ld_out + col) = y1;
+            if (live) *reinterpret_cast<uint2*>(dsc.out1 + (size_t)rw * ld_out + col) = y1;
             if (emit_ssq == 2) {
               a[0] = st_silu(a[0]) * bf16lo_to_f32(y1.x); a[1] = st_silu(a[1]) * bf16hi_to_f32(y1.x);
               a[2] = st_silu(a[2]) * bf16lo_to_f32(y1.y); a[3] = st_silu(a[3]) * bf16hi_to_f32(y1.y);
               // the fp32 product [M][N], for the operation that consumes it
-              if (live) __stcg(reinterpret_cast<float4*>(sp.ws.act + (size_t)rw * __ldg(&op->N) + col), make_float4(a[0], a[1], a[2], a[3]));
+              if (live) __stcg(reinterpret_cast<float4*>(sp.ws.act + (size_t)rw * dsc.N + col), make_float4(a[0], a[1], a[2], a[3]));
             }
           }
           if (emit_ssq != 0) {
@@ -652,46 +808,47 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
               const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
               st_amax_merge(bv, bi, ov, oi);
             }
-            if (lane == 0) __stcg(&sp.ws.cand[(size_t)T * MP + rw], make_float2(bv, __int_as_float(bi)));
-          }
-          named_bar_sync(1, kUnpackThreads);             // all stores of the tile issued; red is free again
-          if (argmax_out != nullptr) {
-            // the CTA that finishes the operation's last tile reduces the per-tile candidates
-            if (tid == 0) {
+            // the warp that stores the row's last candidate reduces the candidates of all tiles
+            int is_last = 0;
+            if (lane == 0) {
+              __stcg(&sp.ws.cand[(size_t)T * MP + rw], make_float2(bv, __int_as_float(bi)));
               int old;
-              asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(sp.ws.amax_done) : "memory");
-              const int is_last = (old == h.n_tiles - 1);
-              if (is_last) *sp.ws.amax_done = 0;
-              s_flag[3] = is_last;
+              asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(sp.ws.status + 16 + rw) : "memory");
+              is_last = (old == h.n_tiles - 1);
+              if (is_last) sp.ws.status[16 + rw] = 0;
             }
-            named_bar_sync(1, kUnpackThreads);
-            if (s_flag[3]) {
-              for (int row = warp; row < sp.M; row += NWG * 4) {
-                float bv = -INFINITY;
-                int bi = 0x7fffffff;
-                for (int tt = lane; tt < h.n_tiles; tt += 32) {
-                  const float2 c = __ldcg(&sp.ws.cand[(size_t)tt * MP + row]);
-                  st_amax_merge(bv, bi, c.x, __float_as_int(c.y));
-                }
-#pragma unroll
-                for (int off = 16; off >= 1; off >>= 1) {
-                  const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-                  const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-                  st_amax_merge(bv, bi, ov, oi);
-                }
-                if (lane == 0) argmax_out[row] = bi;
+            is_last = __shfl_sync(0xffffffffu, is_last, 0);
+            if (is_last && live) {
+              bv = -INFINITY;
+              bi = 0x7fffffff;
+              for (int tt = lane; tt < h.n_tiles; tt += 32) {
+                const float2 c = __ldcg(&sp.ws.cand[(size_t)tt * MP + rw]);
+                st_amax_merge(bv, bi, c.x, __float_as_int(c.y));
               }
+#pragma unroll
+              for (int off = 16; off >= 1; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+                st_amax_merge(bv, bi, ov, oi);
+              }
+              if (lane == 0) argmax_out[rw] = bi;
             }
-            named_bar_sync(1, kUnpackThreads);
           }
-          // the tile is complete: publish it to the operation's counter (one fence after everybody's stores)
-          if (tid == 0 && !(h.flags & kOpNoRelease)) {
-            fence_gpu();
-            red_relaxed_add(&sp.ws.op_done[j], 1);
+          if (pos == end) QL_STAMP(12);
+          // the row of the tile is complete: publish it (one fence after the warp's stores)
+          __syncwarp();
+          if (lane == 0 && !(h.flags & kOpNoRelease)) {
+            if (!(sp.ablate & 16)) fence_gpu();
+            red_relaxed_add(&sp.ws.op_done[((size_t)j * 16 + rw) * kOpDoneStride], 1);
           }
+          if (pos - nch == start) QL_STAMP(6);
+          if (pos == end) QL_STAMP(14);
         }
       }
+      __syncwarp();
+      if (lane == 0) s_prog[warp] = j + 1;
     }
+    QL_CYC_FLUSH();
   }
 
   // every tensor-memory access of the CTA is complete past this barrier
@@ -701,14 +858,18 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
     tc_fence_after_sync();
     tmem_dealloc(tmem, TMEM_COLS);
   }
-  if (tid == 0) {
-    // the last CTA to leave restores the operation counters for the next launch
-    __threadfence();
-    const int old = atomicAdd(sp.ws.exit_cnt, 1);
+  if (warp == 0) {
+    // the last CTA to leave restores the counters for the next launch
+    int old = 0;
+    if (lane == 0) {
+      __threadfence();
+      old = atomicAdd(sp.ws.exit_cnt, 1);
+    }
+    old = __shfl_sync(0xffffffffu, old, 0);
     if (old == (int)gridDim.x - 1) {
-      for (int j = 0; j < sp.n_ops; ++j) sp.ws.op_done[j] = 0;
-      *sp.ws.amax_done = 0;
-      *sp.ws.exit_cnt = 0;
+      for (int i = lane; i < sp.n_ops * 16; i += 32) sp.ws.op_done[(size_t)i * kOpDoneStride] = 0;
+      if (lane < 16) sp.ws.status[16 + lane] = 0;              // per-row arg-max counters
+      if (lane == 0) { *sp.ws.amax_done = 0; *sp.ws.exit_cnt = 0; }
     }
   }
 }
