@@ -228,7 +228,7 @@ int qlinear_stack_w4a16_host(const ql_op* ops, int n_ops,
  * allocator after start-up, a process whose memory budget was handed out before this library was
  * loaded.  Such a caller has its inputs and outputs, but nowhere to put the kernel's scratch
  * (split-K partial tiles, tile counters, arg-max candidates, status word).  Here that scratch is
- * a static device array inside the library, about 5.3 MB, which every GPU that loads the library
+ * a static device array inside the library, about 5.8 MB, which every GPU that loads the library
  * holds until the process exits.  The call allocates nothing and calls nothing that allocates.
  *
  *   arguments as qlinear_w4a16, without the workspace; leading dimensions are K and N

@@ -26,6 +26,8 @@ static std::atomic<int> g_no_release_op{-1};              // test hook: fused op
 static std::atomic<int> g_ablate{0};                      // timing experiments: phases of the stack kernel switched off
 static std::atomic<uint64_t*> g_timeline{nullptr};        // device buffer for the in-kernel timeline (QL_TIMELINE builds)
 
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
 static bool shape_ok(int M, int K, int N, int g) {
   if (M < 1 || M > 64) return false;
   if (g != 64 && g != 128) return false;

@@ -2,11 +2,14 @@
 // tile counters, arg-max candidates, status word) in a static device array of this library
 // instead of a caller-provided workspace.  Nothing is allocated, by this code or by any library
 // it calls.  The kernel is the warp-level MMA kernel of qlinear_w4a16 (QL_PATH_MMA), unchanged.
+#include <atomic>
+
 #include "../../include/qlinear_w4a16.h"
 #include "ql_params.h"
 
 namespace ql {
 cudaError_t launch_linear_mma(LinearParams, cudaStream_t);
+void count_launch();
 
 // Limits of the static variant (stated in the header): M <= 16 rows, N <= 16384 columns.
 constexpr int kStaticMaxM = 16;
@@ -14,7 +17,7 @@ constexpr int kStaticMaxTiles = 128;                          // N <= 128 * 128
 constexpr int kStaticMaxCtas = 160;                           // one CTA per SM
 constexpr size_t kStaticCandBytes = (size_t)kStaticMaxTiles * 16 * 8;
 constexpr size_t kStaticSlotBytes = (size_t)kStaticMaxCtas * 2 * 2 * 16 * kTileN * 4;   // ws_slot_floats(16) floats per slot
-constexpr size_t kStaticBytes = kWsControlBytes + kStaticCandBytes + kStaticSlotBytes;    // about 5.3 MB
+constexpr size_t kStaticBytes = kWsControlBytes + kStaticCandBytes + kStaticSlotBytes;    // about 5.8 MB
 
 // Every GPU that loads the library holds this array until the process exits.
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
@@ -22,15 +25,17 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
 // Device address of the array, resolved once per device.  In host code `g_static_scratch` is only
 // a handle for the runtime, not an address a kernel could use.
 static unsigned char* static_scratch_ptr() {
-  static unsigned char* ptr[16] = {};
+  static std::atomic<unsigned char*> ptr[16] = {};     // two threads may make the first call at once
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 16) return nullptr;
-  if (ptr[dev] == nullptr) {
+  unsigned char* cur = ptr[dev].load(std::memory_order_acquire);
+  if (cur == nullptr) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess) return nullptr;
-    ptr[dev] = static_cast<unsigned char*>(p);
+    cur = static_cast<unsigned char*>(p);
+    ptr[dev].store(cur, std::memory_order_release);
   }
-  return ptr[dev];
+  return cur;
 }
 }  // namespace ql
 
@@ -78,6 +83,7 @@ extern "C" int qlinear_w4a16_static(const void* packed, const uint16_t* X, uint1
   w.n_tiles = kStaticMaxTiles;
   p.ws = w;
   if (launch_linear_mma(p, s) != cudaSuccess) return QL_ERR_CUDA;
+  count_launch();
   return QL_OK;
 }
 

@@ -274,3 +274,72 @@ def test_tolerance_floor_of_bf16_output_rounding():
     print(f"bf16 output-rounding floor: config0 {f0:.3e}, 16x512x1024 {f1:.3e}")
     assert f0 < 2e-3 and f1 < 2e-3
     assert orc.max_scaled_abs_err(orc.round_to_bf16(y1), y1) < 1e-2
+
+
+# ---- the chained layer of the benchmark stack ---------------------------------------------------
+
+def _fraction_to_bf16_bits(v: Fraction) -> int:
+    """Round an exact rational to the nearest bf16 (ties to even), from the format definition
+    (normal range only - enough for this test)."""
+    if v == 0:
+        return 0
+    s = 1 if v < 0 else 0
+    a = -v if s else v
+    e = 0
+    while a >= 2 ** (e + 1):
+        e += 1
+    while a < Fraction(2) ** e:
+        e -= 1
+    q = a / Fraction(2) ** (e - 7)                # in [128, 256)
+    lo = q.numerator // q.denominator
+    rem = q - lo
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and (lo & 1)):
+        lo += 1
+    if lo == 256:
+        lo, e = 128, e + 1
+    assert 1 <= e + 127 <= 254
+    return (s << 15) | ((e + 127) << 7) | (lo - 128)
+
+
+def test_chained_layer_written_out_by_hand():
+    """stack_layer_free_running against the chain spelled out step by step: every linear by the
+    exact-rational brute force, every stored activation rounded to bf16 from the format definition,
+    the glue with scalar Python math.  A wrong slice, gate and up swapped, or a missing rounding
+    between two steps changes the bits."""
+    import math
+    M, hid, q_dim, kv, mlp, g = 2, 16, 8, 4, 32, 8
+    shapes = {"qkv": (hid, q_dim + 2 * kv), "o": (q_dim, hid), "gate": (hid, mlp), "up": (hid, mlp), "down": (mlp, hid)}
+    w = {nm: qsynth.stack_layer_weights(3, nm, g, shapes) for nm in shapes}
+    h = qsynth.stack_h0(M, hid)
+
+    def lin(x_bits, nm):                           # bf16 bits in, bf16 bits out
+        exact = _brute(x_bits, w[nm]["wq"], w[nm]["scale"], w[nm]["zero"], g)
+        return np.array([[_fraction_to_bf16_bits(v) for v in row] for row in exact], dtype=np.uint16)
+
+    def unit(rows):                                # list of rows of Python floats -> bf16 bits
+        out = []
+        for r in rows:
+            rms = math.sqrt(sum(v * v for v in r) / len(r))
+            out.append([_fraction_to_bf16_bits(Fraction(v / rms)) for v in r])
+        return np.array(out, dtype=np.uint16)
+
+    val = lambda bits: [[float(_bf16_fraction(int(b))) for b in row] for row in bits]
+    qkv = lin(h, "qkv")
+    a = unit([r[:q_dim] for r in val(qkv)])        # the q slice stands in for the attention output
+    o = lin(a, "o")
+    r_ = unit(val(o))
+    gt, up = lin(r_, "gate"), lin(r_, "up")
+    prod = [[gv / (1.0 + math.exp(-gv)) * uv for gv, uv in zip(gr, ur)] for gr, ur in zip(val(gt), val(up))]
+    d = unit(prod)
+    dn = lin(d, "down")
+    h_next = unit(val(dn))
+
+    got, ins = orc.stack_layer_free_running(h, w, g, q_dim)
+    assert np.array_equal(ins["qkv"], h) and np.array_equal(ins["o"], a)
+    assert np.array_equal(ins["gate"], r_) and np.array_equal(ins["up"], r_)
+    assert np.array_equal(ins["down"], d)
+    assert np.array_equal(got, h_next)
+    # the variants a plausible mistake would compute are different results
+    swapped = unit([[uv / (1.0 + math.exp(-uv)) * gv for gv, uv in zip(gr, ur)] for gr, ur in zip(val(gt), val(up))])
+    assert not np.array_equal(swapped, d)
+    assert not np.array_equal(unit([r[q_dim - 4:2 * q_dim - 4] for r in val(qkv)]), a)

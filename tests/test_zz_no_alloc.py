@@ -39,6 +39,32 @@ def test_static_scratch_entry_point_matches_workspace_entry_point(ql):
             assert torch.equal(tok, tok_ref)
 
 
+def test_static_scratch_entry_point_g64_and_tokens_only(ql):
+    """Group size 64, and the form that returns only the greedy tokens (Y == NULL); the launch
+    counter of the library counts these calls like any other."""
+    M, K, N, g = 16, 1024, 1280, 64
+    d = qsynth.make_linear([120, 2], M, K, N, g)
+    packed = pack_on_device(ql, d)
+    X = dev_u16(d["x"])
+    ws = ql.new_workspace(M, N)
+    y_ref = torch.zeros((M, N), dtype=torch.int16, device="cuda")
+    tok_ref = torch.zeros((M,), dtype=torch.int32, device="cuda")
+    ql.qlinear_w4a16(packed, X, y_ref, tok_ref, M, K, N, g, ws, path=ql.QL_PATH_MMA)
+    torch.cuda.synchronize()
+    y64 = orc.qlinear_f64(d["x"], d["wq"], d["scale"], d["zero"], g)
+    check_against_oracle(host_u16(y_ref), y64, "workspace entry point, g=64")
+    before = ql.ql_launch_count()
+    for call in range(2):
+        y = torch.full((M, N), 0x7FC0, dtype=torch.int16, device="cuda")
+        ql.qlinear_w4a16_static(packed, X, y, None, M, K, N, g)
+        tok = torch.full((M,), -1, dtype=torch.int32, device="cuda")
+        ql.qlinear_w4a16_static(packed, X, None, tok, M, K, N, g)
+        torch.cuda.synchronize()
+        assert ql.ql_static_status() == ql.QL_OK
+        assert torch.equal(y, y_ref) and torch.equal(tok, tok_ref), f"call {call}"
+    assert ql.ql_launch_count() - before == 4
+
+
 def test_static_scratch_entry_point_rejects_sizes_beyond_its_array(ql):
     P = 0x10000
     lib = ql.load()
