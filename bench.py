@@ -34,9 +34,9 @@ import qsynth  # noqa: E402
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from an ncu capture of a 3-layer launch of the stack kernel:
-# dram read + write = 161.13 MB for 162.32 MB of algorithmic bytes.  Traffic grows in proportion to the
+# dram read + write = 161.78 MB for 162.32 MB of algorithmic bytes.  Traffic grows in proportion to the
 # layers streamed (every packed byte crosses HBM once), so a full launch is scaled by this ratio.
-NCU_TRAFFIC_RATIO = 161.13 / 162.32
+NCU_TRAFFIC_RATIO = 161.78 / 162.32
 
 
 # ------------------------------------------------------------------------------------------------
@@ -156,6 +156,7 @@ class VerifyStep:
                     glue(SU, b["gt"], b["up"], b["d"], mlp), lin("down", b["d"], b["dn"]),
                     glue(U, b["dn"], None, dst, hid)]
         self.h_last = self.h[(n_layers - 1) % 2]
+        self.lm = None
         if lm_head:
             self.lm = device_linear(ql, torch, 999983, hid, qsynth.VOCAB, g)
             ops.append(dict(kind=L, M=M, K=hid, N=qsynth.VOCAB, g=g, ld_in=hid, ld_out=qsynth.VOCAB, packed=self.lm,
@@ -180,6 +181,39 @@ class VerifyStep:
 
     def run_host(self):
         self.ql.qlinear_stack_w4a16_host(self.ops, self.host_in, self.h_in, self.tokens, self.host_tokens, self.ws)
+
+
+def independent_point(ql, torch, M, K, N, g, packed, ws, sym=False, iters=5):
+    """Throughput of one linear shape with cold L2: the distinct weight sets `packed` (together more
+    than twice the L2), one input, DISTINCT outputs, back to back.  Up to 16 rows the whole list
+    is one qlinear_stack_w4a16 call (independent operations: nothing waits for a result); above,
+    qlinear_w4a16 is launched once per weight set.  Returns microseconds per linear and the kernel."""
+    R = len(packed)
+    xin = torch.randn((M, K), device="cuda").to(torch.bfloat16).view(torch.int16)
+    youts = [torch.zeros((M, N), dtype=torch.int16, device="cuda") for _ in range(R)]
+    if M <= 16:
+        ops = ql.make_ops([dict(kind=ql.QL_OP_LINEAR, M=M, K=K, N=N, g=g, ld_in=K, ld_out=N, packed=p, in0=xin, out=y)
+                           for p, y in zip(packed, youts)])
+        plan = ql.ql_stack_plan(ops, ws.data_ptr(), ws.numel())
+        fn = lambda: ql.qlinear_stack_w4a16(ops, ws)
+        kernel = "qstack_tc5_kernel, one stream of chunks" if plan["batch_launches"] else \
+            "qstack_tc5_kernel, every operation split over all SMs, no wait on the predecessor"
+    else:
+        def fn():
+            for p, y in zip(packed, youts):
+                ql.qlinear_w4a16(p, xin, y, None, M, K, N, g, ws)
+        name = ql.PATH_NAMES[ql.ql_select_path(M, K, N, g)]
+        kernel = ("qlinear_tc5_kernel" if name == "tcgen05" else "qlinear_mma_kernel") + ", one launch per linear"
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    ts = sorted(time_events(torch, fn, 1) / R * 1e3 for _ in range(iters))
+    us = ts[len(ts) // 2]
+    b = linear_bytes(M, K, N, g) - ((K // g) * N // 2 if sym else 0)
+    peak, _ = measured_peak()
+    return {"M": M, "K": K, "N": N, "g": g, "zero": "sym8" if sym else "asym", "us": us, "us_min": ts[0], "bytes": b,
+            "GBps": b / us / 1e3, "frac_of_measured_peak": b / us / 1e3 / peak, "frac_of_8TBs": b / us / 1e3 / NOMINAL_HBM_GBS,
+            "kernel": kernel, "weight_sets": R}
 
 
 def max_over_ranks(x: float, world: int, device="cuda") -> float:
@@ -225,6 +259,31 @@ def oracle_sample_seconds(max_layers=12, M=16, g=128, min_seconds=10.0):
         total += time.perf_counter() - t0
         n += 1
     return total, n
+
+
+def oracle_check_last_layer(step, torch):
+    """The configuration that was timed, looked at with the oracle: the five linears of the LAST layer
+    of the step just run (its activation buffers still hold that layer's tensors), each recomputed
+    from the bf16 input the GPU fed it and from the boundary tensors that the oracle's layout
+    reference recovers from the packed weights the kernels streamed.  Part of the CPU-baseline leg."""
+    from oracle import w4a16_oracle as orc
+    step.run()
+    torch.cuda.synchronize()
+    u16 = lambda t: t.cpu().numpy().view(np.uint16)
+    b, l, g = step.bufs, step.n_layers - 1, step.g
+    src = step.h_in if l == 0 else step.h[(l - 1) % 2]
+    feeds = {"qkv": (src, b["qkv"]), "o": (b["a"], b["o"]), "gate": (b["r"], b["gt"]), "up": (b["r"], b["up"]), "down": (b["d"], b["dn"])}
+    worst_rf, worst_me = 0.0, 0.0
+    for nm, (xin, yout) in feeds.items():
+        K, N = qsynth.LAYER_SHAPES[nm]
+        wq, sc, z = orc.unpack_ref(step.packed[l][nm].cpu().numpy(), K, N, g)
+        y64 = orc.qlinear_f64(u16(xin), wq, sc, z, g, col_block=4096)
+        y = orc.bf16_bits_to_f64(u16(yout))
+        worst_rf = max(worst_rf, float(orc.rel_frobenius(y, y64)))
+        worst_me = max(worst_me, float(orc.max_scaled_abs_err(y, y64)))
+    ok = worst_rf <= 2e-3 and worst_me <= 1e-2
+    assert ok, f"timed configuration fails the oracle: relF {worst_rf:.3e}, max scaled error {worst_me:.3e}"
+    return {"layer": l, "linears": 5, "max_rel_frobenius": worst_rf, "max_scaled_abs_err": worst_me, "within_tolerance": ok}
 
 
 def host_threads():
@@ -354,24 +413,45 @@ def run_ours(args, rank, world, local_rank):
                 "traffic": NCU_TRAFFIC_RATIO * total_bytes / launches_per_step,
                 "traffic_source": "ncu capture of a 3-layer launch, scaled by algorithmic bytes",
                 "note": "one step = a chain of 145 dependent fused operations; each waits for the one before it, "
-                        "so the step is bound by dependency latency, not by HBM bandwidth"}
+                        "so the step is bound by dependency latency, not by HBM bandwidth (see single_linear_cold_l2_m16 "
+                        "and lm_head_m16 for the same kernel without the chain)"}
 
-    # ---- the MLP linears on their own (config 1 shapes), cold L2: 36 distinct weight sets back to back ----
-    extras = {}
-    for nm in ("gate", "down", "qkv", "o"):
-        K, N = qsynth.LAYER_SHAPES[nm]
-        xin = torch.randn((M, K), device="cuda").to(torch.bfloat16).view(torch.int16)
-        youts = [torch.zeros((M, N), dtype=torch.int16, device="cuda") for _ in range(step.n_layers)]
-        # independent linears (distinct weights and outputs): the stack launcher lets them overlap
-        ops = ql.make_ops([dict(kind=ql.QL_OP_LINEAR, M=M, K=K, N=N, g=g, ld_in=K, ld_out=N, packed=step.packed[l][nm],
-                                in0=xin, out=youts[l]) for l in range(step.n_layers)])
-        fn = lambda: ql.qlinear_stack_w4a16(ops, step.ws)
-        fn(); fn()
+    # ---- the step's tokens through both entry points must agree ----
+    step.tokens.fill_(-1)
+    step.run()
+    torch.cuda.synchronize()
+    tok_dev = step.tokens.cpu().numpy().copy()
+    step.run_host()
+    tokens_agree = bool(np.array_equal(tok_dev, step.host_tokens.numpy())) if step.lm is not None else None
+    assert tokens_agree is not False, "qlinear_stack_w4a16 and qlinear_stack_w4a16_host returned different tokens"
+
+    # ---- every shape of the step on its own, cold L2: the 36 distinct weight sets of the step, distinct
+    #      outputs, back to back (independent operations) ----
+    extras, sweep_block, lm_point = {}, [], None
+    if step.n_layers >= 24:
+        for nm in ("gate", "down", "qkv", "o"):
+            K, N = qsynth.LAYER_SHAPES[nm]
+            extras[nm] = independent_point(ql, torch, M, K, N, g, [step.packed[l][nm] for l in range(step.n_layers)], step.ws)
+        # configuration 4 in brief (the full 84 points: --sweep): M in {1, 16, 64} x the three shapes, g = 128
+        ws64 = ql.new_workspace(64, qsynth.MLP_DIM)
+        for nm in ("gate", "down", "qkv"):
+            K, N = qsynth.LAYER_SHAPES[nm]
+            for Ms in (1, 16, 64):
+                sweep_block.append(independent_point(ql, torch, Ms, K, N, g, [step.packed[l][nm] for l in range(step.n_layers)],
+                                                     ws64 if Ms > 16 else step.ws, iters=3))
+        del ws64
+    if step.lm is not None:
+        # configuration 3: the LM head with its arg-max on its own (207 MB per call: cold by size)
+        lm_ops = ql.make_ops([dict(kind=ql.QL_OP_LINEAR, M=M, K=qsynth.HIDDEN, N=qsynth.VOCAB, g=g, ld_in=qsynth.HIDDEN,
+                                   ld_out=qsynth.VOCAB, packed=step.lm, in0=step.h_last, out=None, argmax_out=step.tokens)])
+        fn = lambda: ql.qlinear_stack_w4a16(lm_ops, step.ws)
+        for _ in range(3):
+            fn()
         torch.cuda.synchronize()
-        us = time_events(torch, fn, 5) / 5 / step.n_layers * 1e3
-        b = linear_bytes(M, K, N, g)
-        extras[nm] = {"us": us, "GBps": b / us / 1e3, "frac_of_8TBs": b / us / 1e3 / NOMINAL_HBM_GBS,
-                      "path": "tcgen05 (batch kernel)"}
+        ts = sorted(time_events(torch, fn, 1) * 1e3 for _ in range(7))
+        b = linear_bytes(M, qsynth.HIDDEN, qsynth.VOCAB, g, y_bytes=False) + 4 * M
+        lm_point = {"us": ts[len(ts) // 2], "us_min": ts[0], "bytes": b, "GBps": b / ts[len(ts) // 2] / 1e3,
+                    "frac_of_measured_peak": b / ts[len(ts) // 2] / 1e3 / peak, "kernel": "qstack_tc5_kernel (tokens only, no Y)"}
 
     if rank != 0:
         return
@@ -386,13 +466,15 @@ def run_ours(args, rank, world, local_rank):
             "clocks": clocks, "gpu_launches": int(launches), "host_enqueue_ms_per_step": host_enqueue_ms,
             "e2e": {"value": e2e_val, "unit": "GB/s", "h2d_bytes_per_step": int(step.host_in.numel() * 2),
                     "d2h_bytes_per_step": int(step.host_tokens.numel() * 4), "ms_per_step": e2e_s * 1e3},
-            "roofline": roofline, "single_linear_cold_l2_m16": extras}
+            "roofline": roofline, "single_linear_cold_l2_m16": extras, "lm_head_m16": lm_point, "m_sweep": sweep_block,
+            "tokens_agree_device_vs_host_entry": tokens_agree}
     if world == 1 and not args.no_cpu_baseline:
         sec, n_sample = oracle_sample_seconds(12, M, g)
         line["cpu_baseline"] = {"value": per_layer * n_sample / sec / 1e9, "unit": "GB/s", "cores": host_threads(),
                                 "kind": "oracle", "seconds": sec,
                                 "sample": f"layers 0-{n_sample - 1} of the 36-layer stack (M=16, g=128), "
-                                          f"{per_layer * n_sample} algorithmic bytes"}
+                                          f"{per_layer * n_sample} algorithmic bytes",
+                                "timed_run_checked": oracle_check_last_layer(step, torch)}
     print(json.dumps(line), flush=True)
 
 
@@ -408,24 +490,10 @@ def run_sweep(args):
                 packed = [device_linear(ql, torch, 7000 + 100 * si + r, K, N, g, sym) for r in range(reps)]
                 ws = ql.new_workspace(64, N)
                 for M in qsynth.SWEEP_M:
-                    xin = torch.randn((M, K), device="cuda").to(torch.bfloat16).view(torch.int16)
-                    yout = torch.zeros((M, N), dtype=torch.int16, device="cuda")
-                    ops = ql.make_ops([dict(kind=ql.QL_OP_LINEAR, M=M, K=K, N=N, g=g, ld_in=K, ld_out=N, packed=p,
-                                            in0=xin, out=yout) for p in packed])
-                    fn = lambda: ql.qlinear_stack_w4a16(ops, ws)
-                    for _ in range(3):
-                        fn()
-                    torch.cuda.synchronize()
-                    ts = sorted(time_events(torch, fn, 1) / reps * 1e3 for _ in range(10))
-                    plan = ql.ql_stack_plan(ops, ws.data_ptr(), ws.numel())
-                    path = "tcgen05 (persistent stack kernel)" if plan["stack_launches"] else \
-                        ql.PATH_NAMES[ql.ql_select_path(M, K, N, g)] + " (one launch per linear)"
-                    b = linear_bytes(M, K, N, g) - (0 if not sym else (K // g) * N // 2)
-                    us = ts[len(ts) // 2]
-                    print(json.dumps({"sweep": True, "M": M, "K": K, "N": N, "g": g, "zero": "sym8" if sym else "asym",
-                                      "us_median": us, "us_min": ts[0], "bytes": b, "GBps": b / us / 1e3,
-                                      "frac_of_8TBs": b / us / 1e3 / NOMINAL_HBM_GBS, "path": path}), flush=True)
-                del packed
+                    row = independent_point(ql, torch, M, K, N, g, packed, ws, sym=sym, iters=7)
+                    row["sweep"] = True
+                    print(json.dumps(row), flush=True)
+                del packed, ws
                 torch.cuda.empty_cache()
 
 
