@@ -260,7 +260,7 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
       if (batch) {
         uint32_t total = 0;
         for (MegaOp& m : mega) { m.cat_base = total; total += m.total_chunks; }
-        for (MegaOp& m : mega) run_split(total, (uint32_t)ncta, m.nc, m.cq, m.cr);
+        for (MegaOp& m : mega) { run_split(total, (uint32_t)ncta, m.nc, m.cq, m.cr); m.flags |= kOpLazy; }
       } else {
         for (size_t j = 0; j < mega.size(); ++j) {
           MegaOp& m = mega[j];

@@ -36,6 +36,8 @@ struct LinearParams {
 constexpr int kOpDual = 1;        // two matrices (packed0, packed1) share X
 constexpr int kOpWait = 2;        // X may be read only after operation j-1 has finished every tile
 constexpr int kOpWait2 = 8;       // X may be read only after operation j-2 has finished (its partial-tile slots are reused)
+constexpr int kOpLazy = 16;       // nothing in the launch waits for this operation's tiles: they need not be published, and the
+                                  // next tile segment may be started before the current one is finished
 constexpr int kOpNoRelease = 4;   // test hook: finished tiles are not published (the next operation's wait runs out)
 struct MegaOp {
   uint32_t nc, cq, cr;     // CTA i owns run positions [i*cq + i*cr/nc, (i+1)*cq + (i+1)*cr/nc), i < nc

@@ -51,7 +51,8 @@ constexpr int kStMaxStages = 24;
 constexpr uint32_t kStSmemBudget = 232448u;
 constexpr uint32_t kXLbo = 16u * MP + 16u;              // bytes between K-adjacent 8x16-byte core matrices (+16: bank spread)
 __host__ __device__ constexpr uint32_t st_xslot_bytes(int g) { return (uint32_t)(g / 8) * kXLbo; }
-// accumulator exchange buffer + barriers, flags and the two descriptor slots (656 + 64 + 128 + 256 bytes)
+// accumulator exchange buffer + barriers, flags and the two descriptor slots (656 + 64 + 128 + 256 bytes);
+// the table of descriptor heads (32 bytes per operation) follows
 __host__ __device__ constexpr uint32_t st_fixed_smem() { return NWG * MP * 128u * 4u + 2048u; }
 constexpr uint32_t kSlotWords = 2u * MP * 128u;         // floats of one CTA's partial tile, two matrices
 
@@ -88,13 +89,14 @@ __device__ __forceinline__ void fence_gpu() { asm volatile("fence.acq_rel.gpu;" 
 // cycle accounting of the unpack loop (lane 0 of the first warp of every group):
 // 0 wait for the ring stage, 1 wait for a free A buffer, 2 unpack + tensor-memory stores issued, 3 wait::st,
 // 4 wait for the MMAs of the chunk two back, 5 tensor-memory load + scale-accumulate, 6 chunks
-#define QL_CYC_DECL long long cyc_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long cyc_t_ = 0; (void)cyc_t_
-#define QL_CYC_BEGIN() do { cyc_t_ = clock64(); } while (0)
+#define QL_CYC_DECL long long cyc_[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long cyc_te_ = 0; (void)cyc_te_; long long cyc_t_ = clock64(); (void)cyc_t_
+#define QL_CYC_BEGIN() do { const long long now_ = clock64(); cyc_[7] += now_ - cyc_t_; cyc_t_ = now_; } while (0)   /* slot 7: everything else */
 #define QL_CYC_END(i) do { const long long now_ = clock64(); cyc_[i] += now_ - cyc_t_; cyc_t_ = now_; } while (0)
 #define QL_CYC_ADD(i, v) do { cyc_[i] += (v); } while (0)
 #define QL_CYC_FLUSH() do { if (sp.timeline != nullptr && wq == 0 && lane == 0) { \
     uint64_t* dst_ = sp.timeline + (size_t)160 * sp.n_ops * 16 + ((size_t)cta * NWG + w) * 8; \
-    for (int i_ = 0; i_ < 8; ++i_) dst_[i_] = (uint64_t)cyc_[i_]; } } while (0)
+    for (int i_ = 0; i_ < 8; ++i_) dst_[i_] = (uint64_t)cyc_[i_]; \
+    sp.timeline[(size_t)160 * sp.n_ops * 16 + (size_t)2 * 160 * NWG * 8 + (size_t)160 * sp.n_ops + (size_t)cta * NWG + w] = (uint64_t)cyc_te_; } } while (0)
 #define QL_CYC_FLUSH_I() do { if (sp.timeline != nullptr) { \
     uint64_t* dst_ = sp.timeline + (size_t)160 * sp.n_ops * 16 + (size_t)160 * NWG * 8 + ((size_t)cta * NWG + w) * 8; \
     for (int i_ = 0; i_ < 8; ++i_) dst_[i_] = (uint64_t)cyc_[i_]; } } while (0)
@@ -173,9 +175,10 @@ struct OpHead {
   uint32_t nc, cq, cr, cat_base, total_chunks;
   int n_groups, n_tiles, flags;
 };
-__device__ __forceinline__ OpHead load_head(const MegaOp* op) {
-  const uint4 a = __ldg(reinterpret_cast<const uint4*>(op));
-  const uint4 b = __ldg(reinterpret_cast<const uint4*>(op) + 1);
+// (the kernel copies the first 32 bytes of every descriptor into shared memory when it starts)
+__device__ __forceinline__ OpHead load_head(const uint4* s_heads, int j) {
+  const uint4 a = s_heads[2 * j];
+  const uint4 b = s_heads[2 * j + 1];
   OpHead h;
   h.nc = a.x; h.cq = a.y; h.cr = a.z; h.cat_base = a.w;
   h.total_chunks = b.x; h.n_groups = (int)b.y; h.n_tiles = (int)b.z; h.flags = (int)b.w;
@@ -342,8 +345,9 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
   volatile int* s_dep = s_flag + 10;                    // operations whose predecessor is known to be complete
   volatile int* s_invrdy = s_flag + 11;                 // operations whose 1/rms values are in s_inv
   volatile int* s_descrdy = s_flag + 12;                // operations whose descriptor is in s_desc
-  volatile int* s_prog = s_flag + 16;                   // [16] operations each unpack warp has left behind
-  MegaOp* s_desc = reinterpret_cast<MegaOp*>(s_flag + 32);   // [2] descriptors of operations j (slot j & 1), filled by the watcher
+  volatile int* s_prog = s_flag + 16;                   // [16] operations (of those this CTA takes part in) each unpack warp has left behind
+  MegaOp* s_desc = reinterpret_cast<MegaOp*>(s_flag + 32);   // [2] descriptors of the operations this CTA takes part in, filled by the watcher
+  uint4* s_heads = reinterpret_cast<uint4*>(s_desc + 2);     // [n_ops][2] first 32 bytes of every descriptor
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const MegaOp* __restrict__ ops = sp.ops;
@@ -372,6 +376,8 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
     tmem_alloc(s_tmem, TMEM_COLS);
     tmem_relinquish();
   }
+  for (int i = tid; i < 2 * sp.n_ops; i += kStThreads)
+    s_heads[i] = __ldg(reinterpret_cast<const uint4*>(ops + (i >> 1)) + (i & 1));
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -384,7 +390,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
       const uint32_t cb = chunk_bytes(G);
       uint32_t s = 0, ph = 0, gs = 0;
       for (int j = 0; j < sp.n_ops; ++j) {
-        const OpHead h = load_head(ops + j);
+        const OpHead h = load_head(s_heads, j);
         uint32_t start, end;
         op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
         if (start >= end) continue;
@@ -415,28 +421,37 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
     }
   } else if (warp == kWarpWatcher) {
     // ------------------------------------------------------------------ watcher: descriptors, dependencies, row scales
+    int pcount = 0;                                      // operations this CTA took part in so far
     for (int j = 0; j < sp.n_ops; ++j) {
-      // the unpack warps read the descriptor of operation j from shared memory (slot j & 1); the
-      // slot is free once every unpack warp has left operation j-2 behind
-      if (j >= 2) {
+      const OpHead h = load_head(s_heads, j);
+      {
+        // operations this CTA has no chunk of need nothing from it: a later operation it takes part in
+        // waits for its own predecessor, which cannot be complete before everything ahead of it is
+        uint32_t lo, hi;
+        op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, lo, hi);
+        if (lo >= hi) continue;
+      }
+      // the unpack warps read the descriptor from shared memory (two slots, alternating); a slot is
+      // free once every unpack warp has left the operation that used it behind
+      if (pcount >= 2) {
         const uint64_t t0 = globaltimer_ns();
         for (;;) {
           int p = lane < 16 ? s_prog[lane] : 0x7fffffff;
 #pragma unroll
           for (int off = 8; off >= 1; off >>= 1) p = min(p, __shfl_xor_sync(0xffffffffu, p, off));
           p = __shfl_sync(0xffffffffu, p, 0);
-          if (p >= j - 1 || *s_abort) break;
+          if (p >= pcount - 1 || *s_abort) break;
           if (globaltimer_ns() - t0 > wc.budget) { if (lane == 0) wait_fail(wc, 12); break; }
           __nanosleep(64);
         }
       }
-      if (lane < 8) reinterpret_cast<uint4*>(&s_desc[j & 1])[lane] = __ldg(reinterpret_cast<const uint4*>(ops + j) + lane);
+      if (lane < 8) reinterpret_cast<uint4*>(&s_desc[pcount & 1])[lane] = __ldg(reinterpret_cast<const uint4*>(ops + j) + lane);
       __syncwarp();
       if (lane == 0) {
         __threadfence_block();
         *s_descrdy = j + 1;
       }
-      const OpHead h = load_head(ops + j);
+      ++pcount;
       // an operation waits for the one before it (it consumes its output), or only for the one two
       // back (independent operations: the partial-tile slots and flags alternate between two sets)
       const int dep = (h.flags & kOpWait) ? j - 1 : ((h.flags & kOpWait2) ? j - 2 : -1);
@@ -497,7 +512,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
       uint32_t xops = 0;                               // operations this CTA took part in so far
       QL_CYC_DECL;
       for (int j = 0; j < sp.n_ops; ++j) {
-        const OpHead h = load_head(ops + j);
+        const OpHead h = load_head(s_heads, j);
         uint32_t start, end;
         op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
         if (start >= end) continue;
@@ -567,22 +582,18 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
       QL_CYC_END(5);
     };
 
+    int pcount = 0;                                      // operations this CTA took part in so far
     for (int j = 0; j < sp.n_ops; ++j) {
+      const OpHead h = load_head(s_heads, j);
+      uint32_t start, end;
+      op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
+      if (start >= end) continue;
       // the watcher has put the descriptor into shared memory (normally long before)
       if (lane == 0) wait_shared_gt(s_descrdy, j, wc, 13);
       __syncwarp();
       __threadfence_block();
-      const MegaOp& dsc = s_desc[j & 1];
-      OpHead h;
-      h.nc = dsc.nc; h.cq = dsc.cq; h.cr = dsc.cr; h.cat_base = dsc.cat_base;
-      h.total_chunks = dsc.total_chunks; h.n_groups = dsc.n_groups; h.n_tiles = dsc.n_tiles; h.flags = dsc.flags;
-      uint32_t start, end;
-      op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
-      if (start >= end) {
-        __syncwarp();
-        if (lane == 0) s_prog[warp] = j + 1;
-        continue;
-      }
+      const MegaOp& dsc = s_desc[pcount & 1];
+      ++pcount;
       const bool dual = (h.flags & kOpDual) != 0;
       const uint32_t Gn = (uint32_t)h.n_groups;
       const uint32_t my_chunks = end - start;
@@ -679,8 +690,23 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
         if (!(sp.ablate & 1)) {
           if (n_pend == 2) drain(kloc - 2, s_p2);
           if (n_pend >= 1) drain(kloc - 1, s_p1);
+          if (h.flags & kOpLazy) {
+            // nobody waits for this tile: the group's first chunk of the NEXT segment is unpacked
+            // before this segment's tile end, so that its MMAs run while the rows are finished
+            const uint32_t ahead = ((uint32_t)w + NWG - (e % NWG)) % NWG;
+            const bool already = pre_e != 0xffffffffu && pre_e >= e;   // the chunk unpacked before X lies in the next segment
+            if (e + ahead < n_sub_total && !already) {
+              uint32_t s = stg + ahead, ph = sph;
+              if (s >= (uint32_t)NS) { s -= (uint32_t)NS; ph ^= 1; }
+              pre_sc = unpack_subchunk(s, ph);
+              pre_e = e + ahead;
+            }
+          }
         }
         tc_fence_before_sync();
+#ifdef QL_TIMELINE
+        const long long te0_ = clock64();
+#endif
         if (pos == start) QL_STAMP(4);
         if (pos + nch == end) QL_STAMP(8);
 
@@ -837,16 +863,19 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
           if (pos == end) QL_STAMP(12);
           // the row of the tile is complete: publish it (one fence after the warp's stores)
           __syncwarp();
-          if (lane == 0 && !(h.flags & kOpNoRelease)) {
+          if (lane == 0 && !(h.flags & (kOpNoRelease | kOpLazy))) {
             if (!(sp.ablate & 16)) fence_gpu();
             red_relaxed_add(&sp.ws.op_done[((size_t)j * 16 + rw) * kOpDoneStride], 1);
           }
           if (pos - nch == start) QL_STAMP(6);
           if (pos == end) QL_STAMP(14);
         }
+#ifdef QL_TIMELINE
+        cyc_te_ += clock64() - te0_;
+#endif
       }
       __syncwarp();
-      if (lane == 0) s_prog[warp] = j + 1;
+      if (lane == 0) s_prog[warp] = pcount;
     }
     QL_CYC_FLUSH();
   }
@@ -903,7 +932,7 @@ StackPlan stack_plan(const MegaOp* ops, int n_ops, int g, int sms) {
     if (need > n_x) n_x = need;
   }
   const uint32_t stage = align128(chunk_bytes(g)), xslot = st_xslot_bytes(g);
-  const uint32_t fixed = st_fixed_smem();
+  const uint32_t fixed = st_fixed_smem() + 32u * (uint32_t)n_ops;   // + the head table
   if (fixed + n_x * xslot + 6 * stage > kStSmemBudget) return r;
   int ns = (int)((kStSmemBudget - fixed - n_x * xslot) / stage);
   if (ns > kStMaxStages) ns = kStMaxStages;
