@@ -110,6 +110,24 @@ def argmax_rows(y: np.ndarray):
     return idx.astype(np.int64), top1 - top2
 
 
+def accept_prefix(tokens, draft_ids):
+    """Verification of a drafted block (Section 2.2: the target scores the whole block in one pass
+    and keeps the longest prefix of drafted tokens it agrees with; Section 4: under greedy decoding
+    this changes nothing in the output).  tokens[i] is the target's greedy token of row i,
+    draft_ids[i] the drafted token that row i is to confirm.  Returns (a, bonus): a = number of
+    leading rows with tokens[i] == draft_ids[i]; bonus = the target's own token of the first row that
+    disagrees, tokens[a], or -1 if every row agrees (there is no row left to take it from).
+    The paper states the rule in words only; which row confirms which drafted token is the
+    caller's business (it builds draft_ids)."""
+    a = 0
+    for t, d in zip(tokens, draft_ids):
+        if int(t) != int(d):
+            break
+        a += 1
+    bonus = int(tokens[a]) if a < len(tokens) else -1
+    return a, bonus
+
+
 # --------------------------------------------------------------------------------------------
 # the glue that chains linears in the 36-layer benchmark stack (not from the paper: the
 # benchmark's stand-in for normalisation / attention / activation between projections)

@@ -343,3 +343,42 @@ def test_chained_layer_written_out_by_hand():
     swapped = unit([[uv / (1.0 + math.exp(-uv)) * gv for gv, uv in zip(gr, ur)] for gr, ur in zip(val(gt), val(up))])
     assert not np.array_equal(swapped, d)
     assert not np.array_equal(unit([r[q_dim - 4:2 * q_dim - 4] for r in val(qkv)]), a)
+
+
+# ---- verification tail: accepted prefix and bonus token -------------------------------------------
+
+def test_accept_prefix_planted_prefixes_and_brute_force():
+    """Planted agreement prefixes of every length incl. 0, 1, 15 and 16 on a 16-row block; a
+    disagreement later in the block must not matter; and all 2^8 agreement patterns of an 8-row
+    block against the definition 'count leading ones'."""
+    rng = np.random.default_rng(21)
+    tokens = rng.integers(0, 151936, 16)
+    for a in range(17):
+        draft = tokens.copy()
+        if a < 16:
+            draft[a] = (tokens[a] + 7) % 151936                 # first disagreement at row a
+            draft[a + 1:] = rng.integers(0, 151936, 15 - a)     # whatever follows is irrelevant
+            if a + 2 < 16:
+                draft[a + 2] = tokens[a + 2]                    # an agreement after the break does not count
+        got = orc.accept_prefix(tokens, draft)
+        assert got == (a, int(tokens[a]) if a < 16 else -1), (a, got)
+    tok8 = np.arange(100, 108)
+    for pattern in range(256):
+        agree = [(pattern >> i) & 1 for i in range(8)]
+        draft = [int(t) if ok else -5 for t, ok in zip(tok8, agree)]
+        lead = 0
+        while lead < 8 and agree[lead]:
+            lead += 1
+        assert orc.accept_prefix(tok8, draft) == (lead, int(tok8[lead]) if lead < 8 else -1)
+
+
+def test_accept_prefix_uses_the_lowest_index_on_a_logit_tie():
+    """With two equal row maxima the greedy token is the lower index (argmax_rows), and that is the
+    token the drafted id has to match."""
+    y = np.zeros((3, 6))
+    y[0, [2, 4]] = 5.0          # tie -> token 2
+    y[1, 3] = 1.0
+    y[2, 5] = 2.0
+    tokens, _ = orc.argmax_rows(y)
+    assert orc.accept_prefix(tokens, [2, 3, 5]) == (3, -1)
+    assert orc.accept_prefix(tokens, [4, 3, 5]) == (0, 2)
