@@ -158,6 +158,15 @@ int ql_linear_plan(int M, int K, int N, int g, int path, int out[4]);
  *   QL_OP_UNIT_RMS           out[m,:] = bf16( in0[m,:N] / sqrt(mean_n in0[m,n]^2) )      (fp32 math)
  *   QL_OP_SILU_MUL_UNIT_RMS  a = silu(in0) * in1 (fp32);  out[m,:] = bf16( a / sqrt(mean a^2) )
  *
+ * Verification tail (Section 2.2: the target keeps the longest prefix of the drafted block that it
+ * agrees with; Section 4: under greedy decoding the output is unchanged): a LINEAR with argmax_out
+ * may also be given draft_ids[M] and accept_out[2].  The kernel then compares, on the device and
+ * without a host round trip, the greedy token of row i with draft_ids[i], i = 0..M-1, and writes
+ * accept_out[0] = a, the number of leading rows that agree, and accept_out[1] = the greedy token of
+ * row a (the target's own token at the first disagreement), or -1 if all M rows agree.  Which row
+ * confirms which drafted token is the caller's choice (it builds draft_ids; an entry of -1 never
+ * agrees).  M <= 16 only (QL_ERR_UNSUPPORTED otherwise).
+ *
  * in0/in1/out are bf16 with leading dimensions ld_in (in0 and in1) and ld_out, so an operation
  * can read a column slice of a wider tensor.  Operation i sees the results of operations < i.
  * The packed weights of every LINEAR must be complete before the call and must not change while
@@ -191,6 +200,8 @@ typedef struct ql_op {
   const uint16_t* in1;   /* SILU_MUL_UNIT_RMS: second operand */
   uint16_t* out;         /* bf16; LINEAR: may be NULL when argmax_out is given */
   int32_t* argmax_out;   /* LINEAR: [M] or NULL */
+  const int32_t* draft_ids;  /* LINEAR with argmax_out: [M] drafted tokens to verify, or NULL */
+  int32_t* accept_out;       /* with draft_ids: [2] accepted-prefix length, bonus token */
 } ql_op;
 
 int qlinear_stack_w4a16(const ql_op* ops, int n_ops,

@@ -34,6 +34,7 @@ class ql_op(ctypes.Structure):
         ("g", ctypes.c_int32), ("ld_in", ctypes.c_int32), ("ld_out", ctypes.c_int32), ("reserved", ctypes.c_int32),
         ("packed", ctypes.c_void_p), ("in0", ctypes.c_void_p), ("in1", ctypes.c_void_p),
         ("out", ctypes.c_void_p), ("argmax_out", ctypes.c_void_p),
+        ("draft_ids", ctypes.c_void_p), ("accept_out", ctypes.c_void_p),
     ]
 
 
@@ -221,7 +222,7 @@ def make_ops(op_list):
         o.kind = d["kind"]
         o.M, o.K, o.N, o.g = d["M"], d.get("K", 0), d["N"], d.get("g", 0)
         o.ld_in, o.ld_out, o.reserved = d["ld_in"], d["ld_out"], 0
-        for name in ("packed", "in0", "in1", "out", "argmax_out"):
+        for name in ("packed", "in0", "in1", "out", "argmax_out", "draft_ids", "accept_out"):
             t = d.get(name)
             setattr(o, name, None if t is None else (t if isinstance(t, int) else t.data_ptr()))
     return arr

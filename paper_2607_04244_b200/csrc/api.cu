@@ -153,6 +153,7 @@ static MegaOp make_mega(const ql_op& o, const ql_op* second) {
   m.in0 = o.in0; m.in1 = nullptr;
   m.out0 = o.out; m.out1 = second ? second->out : nullptr;
   m.xout = nullptr; m.argmax_out = o.argmax_out;
+  m.draft_ids = o.draft_ids; m.accept_out = o.accept_out;
   m.K = o.K; m.N = o.N; m.ld_in = o.ld_in; m.ld_out = o.ld_out; m.ld_xout = 0;
   m.n_tiles = o.N / kTileN; m.n_groups = o.K / o.g;
   m.total_chunks = (uint32_t)m.n_tiles * (uint32_t)m.n_groups;
@@ -336,6 +337,7 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
         if (st != QL_OK) return st;
       }
       if (!fits) {
+        if (o.draft_ids != nullptr) return QL_ERR_UNSUPPORTED;   // the verification tail lives in the persistent kernel
         int st = flush();
         if (st != QL_OK) return st;
         cnt.single_linears += 1;
@@ -532,9 +534,15 @@ static int validate_stack(const ql_op* ops, int n_ops, const void* workspace, si
       const int st = validate_linear(o.packed, o.in0, o.ld_in, o.out, o.ld_out, o.argmax_out, o.M, o.K, o.N, o.g,
                                      workspace, workspace_bytes);
       if (st != QL_OK) return st;
+      if (o.draft_ids != nullptr || o.accept_out != nullptr) {       // verification tail
+        if (o.draft_ids == nullptr || o.accept_out == nullptr || o.argmax_out == nullptr) return QL_ERR_NULL;
+        if ((reinterpret_cast<uintptr_t>(o.draft_ids) & 3u) || (reinterpret_cast<uintptr_t>(o.accept_out) & 3u)) return QL_ERR_ALIGN;
+        if (o.M > 16) return QL_ERR_UNSUPPORTED;
+      }
     } else if (o.kind == QL_OP_UNIT_RMS || o.kind == QL_OP_SILU_MUL_UNIT_RMS) {
       const int st = validate_glue(o);
       if (st != QL_OK) return st;
+      if (o.draft_ids != nullptr || o.accept_out != nullptr) return QL_ERR_UNSUPPORTED;
     } else {
       return QL_ERR_UNSUPPORTED;
     }

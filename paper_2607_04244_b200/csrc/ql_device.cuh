@@ -15,7 +15,8 @@ __host__ __device__ constexpr uint32_t align128(uint32_t x) { return (x + 127u) 
 
 // ---- workspace layout -----------------------------------------------------------------------
 // [0, 256)        control header: word 0 status, word 1 finished-tile counter (arg-max),
-//                 word 2 finished-CTA counter of the stack kernel, words 16-31 its per-row arg-max counters
+//                 word 2 finished-CTA counter of the stack kernel, words 16-31 its per-row arg-max counters,
+//                 word 32 its counter of rows whose greedy token is final (verification tail)
 // then            per-tile arrival counters (split-K) of the single-linear kernels / partial-row flags of
 //                 the stack kernel                               [kFlagWords]
 // then            per-operation, per-row finished-tile counters of the stack kernel, one 128-byte line each
@@ -31,7 +32,7 @@ constexpr int kMaxTiles = 4096;                   // N <= 128 * 4096
 constexpr int kFlagWords = 8192;                  // tile counters / partial-row flags: [2 parities][160 CTAs][16 rows] fit
 constexpr int kMaxOps = 256;                      // fused operations per stack-kernel launch
 constexpr int kOpDoneStride = 32;                 // ints between the counters of two rows (one line each: they are polled)
-constexpr int kOpDescBytes = 128;
+constexpr int kOpDescBytes = 160;
 constexpr int kWsHeaderBytes = 256;
 constexpr size_t kWsControlBytes = kWsHeaderBytes + (size_t)kFlagWords * 4 + (size_t)kMaxOps * 16 * kOpDoneStride * 4;
 constexpr size_t kWsDescBytes = (size_t)kMaxOps * kOpDescBytes;

@@ -58,6 +58,9 @@ struct MegaOp {
   int prologue;            // 0: X = in0;  1: X = unit_rms(in0);  2: X = unit_rms(silu(in0) * in1)
   int src_tiles;           // column tiles of the producer that make up a normalised row (prologue != 0)
   int emit_ssq;            // 0: none; 1: per-tile row sums of bf16(Y)^2; 2: of (silu(bf16 Y0) * bf16 Y1)^2
+  const int32_t* draft_ids;  // [M] drafted tokens the greedy tokens are compared with (verification tail), else nullptr
+  int32_t* accept_out;       // [2] accepted-prefix length, bonus token
+  uint64_t pad_[2];
 };
 static_assert(sizeof(MegaOp) == kOpDescBytes, "operation descriptor layout");
 

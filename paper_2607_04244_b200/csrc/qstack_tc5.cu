@@ -51,7 +51,7 @@ constexpr int kStMaxStages = 24;
 constexpr uint32_t kStSmemBudget = 232448u;
 constexpr uint32_t kXLbo = 16u * MP + 16u;              // bytes between K-adjacent 8x16-byte core matrices (+16: bank spread)
 __host__ __device__ constexpr uint32_t st_xslot_bytes(int g) { return (uint32_t)(g / 8) * kXLbo; }
-// accumulator exchange buffer + barriers, flags and the two descriptor slots (656 + 64 + 128 + 256 bytes);
+// accumulator exchange buffer + barriers, flags and the two descriptor slots (656 + 64 + 128 + 320 bytes);
 // the table of descriptor heads (32 bytes per operation) follows
 __host__ __device__ constexpr uint32_t st_fixed_smem() { return NWG * MP * 128u * 4u + 2048u; }
 constexpr uint32_t kSlotWords = 2u * MP * 128u;         // floats of one CTA's partial tile, two matrices
@@ -445,7 +445,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
           __nanosleep(64);
         }
       }
-      if (lane < 8) reinterpret_cast<uint4*>(&s_desc[pcount & 1])[lane] = __ldg(reinterpret_cast<const uint4*>(ops + j) + lane);
+      if (lane < (int)(sizeof(MegaOp) / 16)) reinterpret_cast<uint4*>(&s_desc[pcount & 1])[lane] = __ldg(reinterpret_cast<const uint4*>(ops + j) + lane);
       __syncwarp();
       if (lane == 0) {
         __threadfence_block();
@@ -858,6 +858,27 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
                 st_amax_merge(bv, bi, ov, oi);
               }
               if (lane == 0) argmax_out[rw] = bi;
+              // Verification tail: the warp that settles the LAST row's greedy token compares the
+              // block with the drafted tokens - length of the agreeing prefix, and the target's
+              // own token at the first disagreement.
+              if (dsc.draft_ids != nullptr) {
+                int rows_done = 0;
+                if (lane == 0)
+                  asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(rows_done) : "l"(sp.ws.status + 32) : "memory");
+                rows_done = __shfl_sync(0xffffffffu, rows_done, 0);
+                if (rows_done == sp.M - 1) {
+                  const int tok = lane < sp.M ? (lane == rw ? bi : __ldcg(&argmax_out[lane])) : -1;
+                  const int drf = lane < sp.M ? __ldg(&dsc.draft_ids[lane]) : -2;
+                  const unsigned agree = __ballot_sync(0xffffffffu, lane < sp.M && tok == drf);
+                  const int a = __ffs(~agree) - 1;            // first row that disagrees (rows >= M never agree)
+                  const int bonus = __shfl_sync(0xffffffffu, tok, a < sp.M ? a : 0);
+                  if (lane == 0) {
+                    dsc.accept_out[0] = a;
+                    dsc.accept_out[1] = a < sp.M ? bonus : -1;
+                    sp.ws.status[32] = 0;
+                  }
+                }
+              }
             }
           }
           if (pos == end) QL_STAMP(12);
@@ -898,6 +919,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
     if (old == (int)gridDim.x - 1) {
       for (int i = lane; i < sp.n_ops * 16; i += 32) sp.ws.op_done[(size_t)i * kOpDoneStride] = 0;
       if (lane < 16) sp.ws.status[16 + lane] = 0;              // per-row arg-max counters
+      if (lane == 16) sp.ws.status[32] = 0;                    // verification-tail row counter
       if (lane == 0) { *sp.ws.amax_done = 0; *sp.ws.exit_cnt = 0; }
     }
   }

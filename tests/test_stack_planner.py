@@ -135,3 +135,22 @@ def test_stream_k_split_is_balanced_contiguous_and_invertible(ql):
         for c in probes:
             o = lib.ql_plan_chunk_owner(total, ncta, c)
             assert firsts[o] <= c < firsts[o + 1], (total, ncta, c, o)
+
+
+def test_verification_tail_argument_errors(ql):
+    P = 0x100000
+    base = dict(kind=ql.QL_OP_LINEAR, M=16, K=512, N=256, g=128, ld_in=512, ld_out=256, packed=P, in0=P, out=P)
+    wsb = ql.ql_workspace_bytes(64, 256)
+
+    def status(**kw):
+        arr = ql.make_ops([dict(base, **kw)])
+        try:
+            ql.ql_stack_plan(arr, P, wsb)
+            return ql.QL_OK
+        except ql.QlError as e:
+            return e.status
+    assert status(argmax_out=P, draft_ids=P, accept_out=P) == ql.QL_OK
+    assert status(argmax_out=P, draft_ids=P) == ql.QL_ERR_NULL            # accept_out missing
+    assert status(draft_ids=P, accept_out=P) == ql.QL_ERR_NULL            # needs the arg-max
+    assert status(argmax_out=P, draft_ids=P + 2, accept_out=P) == ql.QL_ERR_ALIGN
+    assert status(M=32, argmax_out=P, draft_ids=P, accept_out=P) == ql.QL_ERR_UNSUPPORTED
