@@ -127,7 +127,7 @@ def device_linear(ql, torch, seed, K, N, g, symmetric=False):
 class VerifyStep:
     """Packed weights, activation buffers and the operation list of one verify step."""
 
-    def __init__(self, ql, torch, M=16, g=128, n_layers=qsynth.N_LAYERS, lm_head=True):
+    def __init__(self, ql, torch, M=16, g=128, n_layers=qsynth.N_LAYERS, lm_head=True, symmetric=False):
         self.ql, self.torch, self.M, self.g, self.n_layers = ql, torch, M, g, n_layers
         S = qsynth.LAYER_SHAPES
         hid, mlp, qd = qsynth.HIDDEN, qsynth.MLP_DIM, qsynth.Q_DIM
@@ -139,7 +139,7 @@ class VerifyStep:
         L, U, SU = ql.QL_OP_LINEAR, ql.QL_OP_UNIT_RMS, ql.QL_OP_SILU_MUL_UNIT_RMS
         self.packed, ops = [], []
         for l in range(n_layers):
-            pk = {nm: device_linear(ql, torch, 1000 * l + i, S[nm][0], S[nm][1], g) for i, nm in enumerate(S)}
+            pk = {nm: device_linear(ql, torch, 1000 * l + i, S[nm][0], S[nm][1], g, symmetric) for i, nm in enumerate(S)}
             self.packed.append(pk)
             src = self.h_in if l == 0 else self.h[(l - 1) % 2]
             dst = self.h[l % 2]
@@ -478,6 +478,42 @@ def run_ours(args, rank, world, local_rank):
     print(json.dumps(line), flush=True)
 
 
+def run_drafter(args):
+    """Second workload (paper Sections 3.2, 3.3): the drafter's W4 linears - 5 layers, hidden 2560,
+    group-wise symmetric INT4 with groups of 128 (zero == NULL at the boundary), M = 16 - through
+    the same launcher.  The projection widths are SYNTHETIC (the target's; the paper does not give
+    them).  One step streams 0.27 GB, which fits in L2, so a buffer larger than L2 is written
+    between steps.  Prints one JSON line."""
+    import torch
+    import paper_2607_04244_b200 as ql
+    ql.load()
+    M, g, L = 16, 128, qsynth.DRAFTER_LAYERS
+    step = VerifyStep(ql, torch, M, g, n_layers=L, lm_head=False, symmetric=True)
+    per_layer = sum(linear_bytes(M, K, N, g) - (K // g) * N // 2 for (K, N) in qsynth.LAYER_SHAPES.values())   # no zero points
+    total = L * per_layer
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    for _ in range(max(args.warmup, 3)):
+        step.run()
+    torch.cuda.synchronize()
+    assert ql.ql_device_status(step.ws) == ql.QL_OK
+    ts = []
+    for _ in range(args.steps):
+        flush.fill_(1)
+        ts.append(time_events(torch, step.run, 1))
+    ms = float(np.median(ts))
+    peak, peak_kind = measured_peak()
+    val = total / (ms * 1e-3) / 1e9
+    print(json.dumps({"metric": "W4A16 drafter-block HBM GB/s at M=16 (5 symmetric-INT4 layers per step)", "value": val,
+                      "unit": "GB/s", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+                      "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": "drafter_block: 5 layers x (qkv, o, gate, up, down), symmetric g=128, M=16, "
+                                             "synthetic widths (the target's)", "algorithmic_bytes_per_step": total,
+                                 "l2": "256 MB written between steps (the step's 0.27 GB would otherwise stay in L2)"},
+                      "roofline": {"bound": "hbm", "achieved": val, "peak": peak, "unit": "GB/s", "frac": val / peak,
+                                   "peak_kind": f"of {peak_kind}", "kernel": "qstack_tc5_kernel"},
+                      "gpu_launches": args.steps + max(args.warmup, 3)}), flush=True)
+
+
 def run_sweep(args):
     """M-sweep: M x three shapes x g in {64,128} x zero mode; one JSON line per point."""
     import torch
@@ -563,6 +599,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--workload", default="verify_step", choices=["verify_step", "drafter"],
+                    help="drafter: the second workload (5 symmetric-INT4 layers, synthetic widths)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=qsynth.N_LAYERS,
                     help="layers of the stack (default: the full 36; smaller values are for profiler captures)")
@@ -577,6 +615,9 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank, world)
+        return
+    if args.workload == "drafter":
+        run_drafter(args)
         return
     if args.sweep:
         run_sweep(args)

@@ -110,6 +110,28 @@ def argmax_rows(y: np.ndarray):
     return idx.astype(np.int64), top1 - top2
 
 
+def requant_codes(w_bits: np.ndarray, scale_bits: np.ndarray, zero: np.ndarray | None, g: int) -> np.ndarray:
+    """Grid-preserving re-quantisation (Section 2.1: after distillation the updated BF16 weights are
+    rounded back onto the same quantisation grid, which gives new INT4 codes under the original
+    frozen scales).  For bf16 weights w[K,N], the frozen bf16 scales s[K/g,N] and zero points z
+    (None: the symmetric grid, z = 8):
+        code[k,n] = clamp( rne( float32(w[k,n]) / float32(s[k div g, n]) ) + z[k div g, n], 0, 15 )
+    The quotient is the IEEE float32 division (correctly rounded), rne is round-half-to-even to an
+    integer: the paper fixes neither, this is the precision the decision is taken in on both sides.
+    Returns uint8 codes [K, N]."""
+    w = bf16_bits_to_f64(w_bits).astype(np.float32)           # exact widening
+    s = bf16_bits_to_f64(scale_bits).astype(np.float32)
+    K, N = w.shape
+    ng = K // g
+    z = np.full((ng, N), 8, dtype=np.int64) if zero is None else zero.astype(np.int64)
+    q = np.empty((K, N), dtype=np.uint8)
+    for G in range(ng):
+        quo = w[G * g:(G + 1) * g, :] / s[G:G + 1, :]           # float32 / float32 -> float32
+        r = np.rint(quo).astype(np.int64)                        # half to even
+        q[G * g:(G + 1) * g, :] = np.clip(r + z[G:G + 1, :], 0, 15).astype(np.uint8)
+    return q
+
+
 def accept_prefix(tokens, draft_ids):
     """Verification of a drafted block (Section 2.2: the target scores the whole block in one pass
     and keeps the longest prefix of drafted tokens it agrees with; Section 4: under greedy decoding

@@ -113,6 +113,19 @@ def stack_layer_weights(layer: int, name: str, g: int = 128, shapes: dict | None
     return make_linear([layer, LINEAR_IDX[name]], 0, K, N, g, with_x=False)
 
 
+# Second workload: the drafter.  The paper gives its depth (5 layers), hidden size (2560), block
+# size (16) and quantisation (group-wise symmetric INT4, groups of 128) but not its projection
+# widths; the widths used here are the target's (SYNTHETIC: 5 x 100.9 M = 505 M parameters, close to
+# the ~537 M the paper states for the whole drafter).
+DRAFTER_LAYERS = 5
+
+
+def drafter_layer_weights(layer: int, name: str, g: int = 128, shapes: dict | None = None) -> dict:
+    """Weights of one projection of one drafter layer: symmetric codes (zero point 8), entropy [5, layer, linear_idx]."""
+    K, N = (shapes or LAYER_SHAPES)[name]
+    return make_linear([5, layer, LINEAR_IDX[name]], 0, K, N, g, symmetric=True, with_x=False)
+
+
 def stack_h0(M: int = 16, hidden: int = HIDDEN) -> np.ndarray:
     """Input of layer 0 of the stack: bf16 N(0,1) [M, hidden], entropy [2, 0xACE]."""
     return make_x([2, 0xACE], M, hidden)

@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 NAMES = ("qkv", "o", "gate", "up", "down")
 
 
-def build_stack(ql, n_layers, shapes, M, g, q_dim, layer_ids=None, lm_head=None):
+def build_stack(ql, n_layers, shapes, M, g, q_dim, layer_ids=None, lm_head=None, drafter=False):
     """Allocates activations, packs weights and returns (ops list, buffers, weights per layer)."""
     hid = shapes["qkv"][0]
     mlp = shapes["gate"][1]
@@ -27,8 +27,9 @@ def build_stack(ql, n_layers, shapes, M, g, q_dim, layer_ids=None, lm_head=None)
     L, U, SU = ql.QL_OP_LINEAR, ql.QL_OP_UNIT_RMS, ql.QL_OP_SILU_MUL_UNIT_RMS
     for l in range(n_layers):
         lid = l if layer_ids is None else layer_ids[l]
-        w = {nm: qsynth.stack_layer_weights(lid, nm, g, shapes) for nm in NAMES}
-        pk = {nm: pack_on_device(ql, w[nm]) for nm in NAMES}
+        gen = qsynth.drafter_layer_weights if drafter else qsynth.stack_layer_weights
+        w = {nm: gen(lid, nm, g, shapes) for nm in NAMES}
+        pk = {nm: pack_on_device(ql, w[nm], zero_none=drafter) for nm in NAMES}   # symmetric: no zero points passed
         weights.append(w)
         packed_all.append(pk)
 
@@ -115,6 +116,23 @@ def test_full_size_layers_teacher_forced(ql):
     torch.cuda.synchronize()
     assert ql.ql_device_status(ws) == ql.QL_OK
     for l in range(3):
+        check_layer(l, bufs, weights, qsynth.LAYER_SHAPES, g, qsynth.Q_DIM)
+
+
+def test_drafter_layers_symmetric_full_size(ql):
+    """The second workload: drafter layers (group-wise symmetric INT4, groups of 128, M = 16; paper
+    Sections 3.2 and 3.3) through the same launcher, zero == NULL at the boundary.  Two of the five
+    layers at full (synthetic) widths, chained, every linear checked teacher-forced."""
+    M, g = 16, 128
+    ops, bufs, weights, _pk = build_stack(ql, 2, qsynth.LAYER_SHAPES, M, g, qsynth.Q_DIM, layer_ids=[0, 4], drafter=True)
+    bufs["h"][0].copy_(dev_u16(qsynth.stack_h0(M)))
+    ws = ql.new_workspace(M, qsynth.MLP_DIM)
+    arr = ql.make_ops(ops)
+    ql.qlinear_stack_w4a16(arr, ws)
+    torch.cuda.synchronize()
+    assert ql.ql_device_status(ws) == ql.QL_OK
+    assert all(np.all(w[nm]["zero"] == 8) for w in weights for nm in NAMES)
+    for l in range(2):
         check_layer(l, bufs, weights, qsynth.LAYER_SHAPES, g, qsynth.Q_DIM)
 
 

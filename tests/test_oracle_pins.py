@@ -382,3 +382,75 @@ def test_accept_prefix_uses_the_lowest_index_on_a_logit_tie():
     tokens, _ = orc.argmax_rows(y)
     assert orc.accept_prefix(tokens, [2, 3, 5]) == (3, -1)
     assert orc.accept_prefix(tokens, [4, 3, 5]) == (0, 2)
+
+
+# ---- grid-preserving re-quantisation ---------------------------------------------------------------
+
+def _fraction_to_f32(v: Fraction) -> Fraction:
+    """Exact rational -> nearest IEEE float32 (ties to even), as an exact rational; normal range."""
+    if v == 0:
+        return Fraction(0)
+    s, a, e = (-1 if v < 0 else 1), abs(v), 0
+    while a >= 2 ** (e + 1):
+        e += 1
+    while a < Fraction(2) ** e:
+        e -= 1
+    q = a / Fraction(2) ** (e - 23)
+    lo = q.numerator // q.denominator
+    rem = q - lo
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and (lo & 1)):
+        lo += 1
+    return s * lo * Fraction(2) ** (e - 23)
+
+
+def _rne_int(v: Fraction) -> int:
+    lo = v.numerator // v.denominator               # floor
+    rem = v - lo
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and (lo & 1)):
+        lo += 1
+    return lo
+
+
+def test_requant_brute_force_exact_rationals():
+    """Every element by exact rational arithmetic: the quotient rounded to float32 from its exact
+    value, then to the nearest integer with ties to even, shifted by the zero point and clamped."""
+    rng = np.random.default_rng(31)
+    K, N, g = 32, 6, 16
+    scale = qsynth.f32_to_bf16_bits(np.abs(rng.standard_normal((K // g, N), dtype=np.float32)) * np.float32(0.01) + np.float32(1e-3))
+    zero = rng.integers(0, 16, (K // g, N), dtype=np.uint8)
+    w = qsynth.f32_to_bf16_bits(rng.standard_normal((K, N), dtype=np.float32) * np.float32(0.08))
+    for z in (zero, None):
+        got = orc.requant_codes(w, scale, z, g)
+        for k in range(K):
+            for n in range(N):
+                quo = _fraction_to_f32(_bf16_fraction(int(w[k, n])) / _bf16_fraction(int(scale[k // g, n])))
+                zz = 8 if z is None else int(z[k // g, n])
+                want = min(15, max(0, _rne_int(quo) + zz))
+                assert int(got[k, n]) == want, (k, n)
+
+
+def test_requant_hand_made_grid_ties_and_clamps():
+    """Scale 2^-3, zero point 5: weights placed exactly on the grid come back as their codes; exact
+    halves go to the even neighbour; values beyond the grid clamp to 0 and 15."""
+    g = 8
+    s = np.full((1, 1), 0x3E00, dtype=np.uint16)                # 2^-3
+    z = np.full((1, 1), 5, dtype=np.uint8)
+    vals = [(c - 5) / 8 for c in range(8)]                      # on the grid: codes 0..7
+    w = qsynth.f32_to_bf16_bits(np.array(vals, dtype=np.float32).reshape(8, 1))
+    assert orc.requant_codes(w, s, z, g)[:, 0].tolist() == list(range(8))
+    halves = [0.5 / 8, 1.5 / 8, 2.5 / 8, -0.5 / 8, -1.5 / 8, 100.0, -100.0, 9.5 / 8]
+    w = qsynth.f32_to_bf16_bits(np.array(halves, dtype=np.float32).reshape(8, 1))
+    #            0.5->0   1.5->2   2.5->2   -0.5->-0  -1.5->-2  clamp  clamp  9.5->10
+    assert orc.requant_codes(w, s, z, g)[:, 0].tolist() == [5, 7, 7, 5, 3, 15, 0, 15]
+
+
+def test_requant_round_trip_of_dequantised_weights_with_power_of_two_scales():
+    """With power-of-two scales the dequantised weights are exact in bf16, so re-quantising them
+    returns the codes they came from (the grid is preserved)."""
+    rng = np.random.default_rng(32)
+    K, N, g = 64, 16, 32
+    codes = rng.integers(0, 16, (K, N), dtype=np.uint8)
+    zero = rng.integers(0, 16, (K // g, N), dtype=np.uint8)
+    scale = np.full((K // g, N), 0x3D00, dtype=np.uint16)       # 2^-5
+    w = orc.dequant_f32(qsynth.pack_codes_k8(codes), scale, zero, g)
+    assert np.array_equal(orc.requant_codes(qsynth.f32_to_bf16_bits(w), scale, zero, g), codes)
