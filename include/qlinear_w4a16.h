@@ -112,6 +112,21 @@ int qpack_w4_g128(const uint32_t* wq, const uint16_t* scale, const uint8_t* zero
                   int K, int N, int g, void* packed, size_t packed_bytes, void* stream);
 
 /*
+ * qrequant_pack_w4 - grid-preserving re-quantisation, fused with the repack (Section 2.1: after
+ * distillation the updated BF16 weights are rounded back onto the same quantisation grid, which
+ * gives new INT4 codes under the original, frozen scales).
+ *
+ *   w       [K, N] bf16 bit patterns, row-major: the updated weights
+ *   scale   [K/g, N] bf16, zero [K/g, N] or NULL (z == 8): the frozen grid, as in qpack_w4_g128
+ *   packed  out, ql_packed_bytes(K,N,g) bytes: the layout of qpack_w4_g128, holding the codes
+ *           clamp( rne( float32(w) / float32(scale) ) + zero, 0, 15 )
+ * The quotient is the IEEE float32 division, rne rounds halves to the even integer: the result
+ * is fully determined (bit-exact against the reference).  Errors as qpack_w4_g128.
+ */
+int qrequant_pack_w4(const uint16_t* w, const uint16_t* scale, const uint8_t* zero,
+                     int K, int N, int g, void* packed, size_t packed_bytes, void* stream);
+
+/*
  * qlinear_w4a16 - Y = X * dequant(packed)  (Section 2.1's s (.) W_q applied to a block of M
  * drafted tokens, Section 2.2), optionally followed by the greedy token of each row (Section 4).
  *

@@ -22,7 +22,7 @@ QL_OP_LINEAR, QL_OP_UNIT_RMS, QL_OP_SILU_MUL_UNIT_RMS = 0, 1, 2
 EXPORTS = [
     "ql_status_str", "ql_packed_bytes", "ql_workspace_bytes", "ql_workspace_init", "ql_device_status",
     "ql_device_status_raw",
-    "qpack_w4_g128", "qlinear_w4a16", "qlinear_w4a16_path", "ql_select_path", "qlinear_stack_w4a16",
+    "qpack_w4_g128", "qrequant_pack_w4", "qlinear_w4a16", "qlinear_w4a16_path", "ql_select_path", "qlinear_stack_w4a16",
     "qlinear_stack_w4a16_host", "ql_launch_count", "qlinear_w4a16_static", "ql_static_status", "ql_stack_plan", "ql_linear_plan", "ql_plan_first_chunk", "ql_plan_chunk_owner",
     "ql_debug_set_wait_budget_ns", "ql_debug_no_release", "ql_debug_set_timeline", "ql_debug_timeline_enabled", "ql_debug_set_ablate",
 ]
@@ -73,6 +73,8 @@ def load(path: str | None = None):
     lib.ql_device_status_raw.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
     lib.qpack_w4_g128.restype = i32
     lib.qpack_w4_g128.argtypes = [vp, vp, vp, i32, i32, i32, vp, sz, vp]
+    lib.qrequant_pack_w4.restype = i32
+    lib.qrequant_pack_w4.argtypes = [vp, vp, vp, i32, i32, i32, vp, sz, vp]
     lib.qlinear_w4a16.restype = i32
     lib.qlinear_w4a16.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, sz, vp]
     lib.qlinear_w4a16_path.restype = i32
@@ -201,6 +203,17 @@ def qpack_w4_g128(wq, scale, zero, K: int, N: int, g: int, packed=None, stream=N
         packed = torch.empty(ql_packed_bytes(K, N, g), dtype=torch.uint8, device=wq.device)
     _check(load().qpack_w4_g128(wq.data_ptr(), scale.data_ptr(), _ptr(zero), K, N, g, packed.data_ptr(),
                                 packed.numel(), _stream(stream)), "qpack_w4_g128")
+    return packed
+
+
+def qrequant_pack_w4(w, scale, zero, K: int, N: int, g: int, packed=None, stream=None):
+    """w int16 (bf16 bits) [K,N], scale int16 (bf16 bits) [K/g,N], zero uint8 [K/g,N] or None.
+    Returns the packed uint8 tensor holding the re-quantised codes."""
+    import torch
+    if packed is None:
+        packed = torch.empty(ql_packed_bytes(K, N, g), dtype=torch.uint8, device=w.device)
+    _check(load().qrequant_pack_w4(w.data_ptr(), scale.data_ptr(), _ptr(zero), K, N, g, packed.data_ptr(),
+                                   packed.numel(), _stream(stream)), "qrequant_pack_w4")
     return packed
 
 

@@ -9,6 +9,7 @@
 
 namespace ql {
 cudaError_t launch_qpack(const uint32_t*, const uint16_t*, const uint8_t*, int, int, int, uint8_t*, cudaStream_t);
+cudaError_t launch_qrequant(const uint16_t*, const uint16_t*, const uint8_t*, int, int, int, uint8_t*, cudaStream_t);
 cudaError_t launch_linear_mma(LinearParams, cudaStream_t);
 size_t plan_linear_mma(LinearParams&);
 cudaError_t launch_linear_tc5(LinearParams, int sms, cudaStream_t, bool pdl);
@@ -464,6 +465,18 @@ int qpack_w4_g128(const uint32_t* wq, const uint16_t* scale, const uint8_t* zero
   if (!aligned16(wq) || !aligned16(scale) || !aligned16(packed)) return QL_ERR_ALIGN;
   if (packed_bytes < ql_packed_bytes(K, N, g)) return QL_ERR_WORKSPACE;
   if (launch_qpack(wq, scale, zero, K, N, g, static_cast<uint8_t*>(packed), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return QL_ERR_CUDA;
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return QL_OK;
+}
+
+int qrequant_pack_w4(const uint16_t* w, const uint16_t* scale, const uint8_t* zero, int K, int N, int g, void* packed,
+                     size_t packed_bytes, void* stream) {
+  if (w == nullptr || scale == nullptr || packed == nullptr) return QL_ERR_NULL;
+  if (!shape_ok(1, K, N, g)) return QL_ERR_SHAPE;
+  if (!aligned16(w) || !aligned16(scale) || !aligned16(packed)) return QL_ERR_ALIGN;
+  if (packed_bytes < ql_packed_bytes(K, N, g)) return QL_ERR_WORKSPACE;
+  if (launch_qrequant(w, scale, zero, K, N, g, static_cast<uint8_t*>(packed), static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return QL_ERR_CUDA;
   g_launches.fetch_add(1, std::memory_order_relaxed);
   return QL_OK;
