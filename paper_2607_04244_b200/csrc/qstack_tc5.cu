@@ -642,13 +642,20 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
 
       // -------- the group's first chunk of the operation is unpacked BEFORE its X exists (the A
       //          operand depends on weights only; the issuer holds the MMAs back) --------
+      // this group's sub-chunks of the operation are e = w, w + 4, ...; (s_own, ph_own) is the ring
+      // stage and phase of the next one
+      uint32_t e_own = (uint32_t)w, s_own = stg + (uint32_t)w, ph_own = sph;
+      if (s_own >= (uint32_t)NS) { s_own -= (uint32_t)NS; ph_own ^= 1; }
+      auto advance_own = [&]() {
+        e_own += NWG;
+        s_own += NWG;
+        if (s_own >= (uint32_t)NS) { s_own -= (uint32_t)NS; ph_own ^= 1; }
+      };
       float pre_sc = 0.f;
-      uint32_t pre_e = 0xffffffffu;                     // sub-chunk of this group that is already unpacked
-      if ((uint32_t)w < n_sub_total && !(sp.ablate & 1)) {
-        uint32_t s = stg + (uint32_t)w, ph = sph;
-        if (s >= (uint32_t)NS) { s -= (uint32_t)NS; ph ^= 1; }
-        pre_sc = unpack_subchunk(s, ph);
-        pre_e = (uint32_t)w;
+      bool pre_done = false;                            // sub-chunk e_own is already unpacked
+      if (e_own < n_sub_total && !(sp.ablate & 1)) {
+        pre_sc = unpack_subchunk(s_own, ph_own);
+        pre_done = true;
       }
       QL_STAMP(1);
       // -------- X duty (all 512 threads): wait for the previous operation, build the X operand --------
@@ -656,7 +663,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
       QL_STAMP(3);
 
       // -------- chunks of this operation --------
-      uint32_t pos = start, e = 0;                      // e: sub-chunk counter of the operation (this CTA)
+      uint32_t pos = start, e_seg_end = 0;              // sub-chunks of the operation up to the end of the current segment
       while (pos < end) {
         const uint32_t T = pos / Gn;
         const uint32_t g0 = pos - T * Gn;
@@ -667,40 +674,33 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
         // before this chunk's tensor-memory stores are issued: a tcgen05.ld queued behind them waits
         int n_pend = 0;
         float s_p1 = 0.f, s_p2 = 0.f;
-        const uint32_t n_sub = nch * (dual ? 2u : 1u);
-        for (uint32_t si = 0; si < n_sub; ++si, ++e) {
-          const uint32_t my_stage = stg, my_phase = sph;
-          if (++stg == (uint32_t)NS) { stg = 0; sph ^= 1; }
-          if ((int)(e % NWG) != w) continue;
+        e_seg_end += nch * (dual ? 2u : 1u);
+        while (e_own < e_seg_end) {
           float sc;
           if (sp.ablate & 1) {
             sc = 0.f;
-          } else if (e == pre_e) {
+          } else if (pre_done) {
             sc = pre_sc;                                 // unpacked ahead (before X duty, or before the previous tile end)
+            pre_done = false;
           } else {
             if (n_pend == 2) { drain(kloc - 2, s_p2); n_pend = 1; }
-            sc = unpack_subchunk(my_stage, my_phase);
+            sc = unpack_subchunk(s_own, ph_own);
           }
           if (sp.ablate & 1) n_pend = 0;
           s_p2 = s_p1;
           s_p1 = sc;
           ++n_pend;
           ++kloc;
+          advance_own();
         }
         if (!(sp.ablate & 1)) {
           if (n_pend == 2) drain(kloc - 2, s_p2);
           if (n_pend >= 1) drain(kloc - 1, s_p1);
-          if (h.flags & kOpLazy) {
-            // nobody waits for this tile: the group's first chunk of the NEXT segment is unpacked
-            // before this segment's tile end, so that its MMAs run while the rows are finished
-            const uint32_t ahead = ((uint32_t)w + NWG - (e % NWG)) % NWG;
-            const bool already = pre_e != 0xffffffffu && pre_e >= e;   // the chunk unpacked before X lies in the next segment
-            if (e + ahead < n_sub_total && !already) {
-              uint32_t s = stg + ahead, ph = sph;
-              if (s >= (uint32_t)NS) { s -= (uint32_t)NS; ph ^= 1; }
-              pre_sc = unpack_subchunk(s, ph);
-              pre_e = e + ahead;
-            }
+          // nobody waits for this tile: the group's first chunk of the NEXT segment is unpacked
+          // before this segment's tile end, so that its MMAs run while the rows are finished
+          if ((h.flags & kOpLazy) && e_own < n_sub_total && !pre_done) {
+            pre_sc = unpack_subchunk(s_own, ph_own);
+            pre_done = true;
           }
         }
         tc_fence_before_sync();
@@ -894,6 +894,11 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
 #ifdef QL_TIMELINE
         cyc_te_ += clock64() - te0_;
 #endif
+      }
+      {
+        const uint32_t t = stg + n_sub_total;             // ring position after this operation's sub-chunks
+        sph ^= (t / (uint32_t)NS) & 1u;
+        stg = t % (uint32_t)NS;
       }
       __syncwarp();
       if (lane == 0) s_prog[warp] = pcount;
