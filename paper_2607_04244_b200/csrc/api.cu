@@ -83,6 +83,7 @@ static int prepare_linear(LinearParams& p, const void* packed, const uint16_t* X
   p.ncta = ncta;
   p.m_pad = m_pad;
   p.n_stages = 0; p.stage_bytes = 0; p.n_x = 0; p.x_phase = 0;
+  p.ablate = g_ablate.load(std::memory_order_relaxed);
   p.ws = ws_carve(workspace, n_tiles, m_pad);
   return QL_OK;
 }

@@ -22,6 +22,7 @@ struct LinearParams {
   int n_x;                 // X slots (groups) in shared memory per CTA
   int x_phase;             // 0: X resident; P > 0: X of the next P chunks reloaded every P chunks
   uint32_t stage_bytes;    // bytes of one ring stage (weights chunk + X slice)
+  int ablate;              // timing experiments (1: chunks are received but not computed)
   Workspace ws;
 };
 

@@ -21,13 +21,14 @@
 
 namespace ql {
 
-constexpr int kMmaThreads = 288;
+constexpr int kMmaMaxThreads = 544;                     // 4 k-groups of 4 warps + the producer warp
+__host__ __device__ constexpr int mma_kgroups(int mt) { return mt == 1 ? 4 : 2; }   // k-groups (sets of 4 consumer warps taking alternate chunks)
 constexpr int kMaxStages = 32;
 constexpr uint32_t kSmemBudget = 232448u;   // 227 KB of dynamic shared memory per CTA
 
 __host__ __device__ inline uint32_t mma_stage_bytes(int g) { return align128(chunk_bytes(g)); }
 __host__ __device__ inline uint32_t mma_xslot_bytes(int g, int m_pad) { return (uint32_t)m_pad * 2u * g; }
-__host__ __device__ inline uint32_t mma_fixed_smem(int mt) { return 8192u * mt + kMaxStages * 16u + 2048u + 64u; }
+__host__ __device__ inline uint32_t mma_fixed_smem(int mt) { return 8192u * mt * (mma_kgroups(mt) - 1) + kMaxStages * 16u + 2048u + 64u; }
 
 // k-permutation used inside a 32-row block c of a group (it only has to be the same for X and W):
 // lane t = lane & 3 owns rows 32c + 8t + i, i = 0..7; the first MMA of the pair contracts
@@ -102,7 +103,9 @@ __device__ __forceinline__ void amax_merge(float& bv, int& bi, float v, int i) {
 }
 
 template <int MT, int G>
-__global__ void __launch_bounds__(kMmaThreads, 1) qlinear_mma_kernel(const __grid_constant__ LinearParams p) {
+__global__ void __launch_bounds__(mma_kgroups(MT) * 128 + 32, 1) qlinear_mma_kernel(const __grid_constant__ LinearParams p) {
+  constexpr int KG = mma_kgroups(MT);
+  constexpr int NCONS = KG * 128;                        // consumer threads
   extern __shared__ __align__(1024) uint8_t smem[];
   const int NS = p.n_stages;
   const uint32_t stage = p.stage_bytes;
@@ -111,7 +114,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qlinear_mma_kernel(const __gri
   const uint32_t xslot = mma_xslot_bytes(G, p.m_pad);
   uint8_t* after_x = xbuf + (size_t)p.n_x * xslot;
   float4* red4 = reinterpret_cast<float4*>(after_x);
-  uint64_t* full = reinterpret_cast<uint64_t*>(after_x + 8192u * MT);
+  uint64_t* full = reinterpret_cast<uint64_t*>(after_x + 8192u * MT * (KG - 1));
   uint64_t* empty = full + kMaxStages;
   float2* s_amax = reinterpret_cast<float2*>(empty + kMaxStages);      // [4][64]
   int* s_flag = reinterpret_cast<int*>(s_amax + 4 * 64);                // [0..3] flags, [8] abort
@@ -133,7 +136,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qlinear_mma_kernel(const __gri
   }
   __syncthreads();
 
-  if (warp == 8) {
+  if (warp == KG * 4) {
     // ------------------------------------------------------------------ producer
     uint32_t it = 0;
     if (lane == 0) {
@@ -176,7 +179,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qlinear_mma_kernel(const __gri
   auto load_x_slots = [&](uint32_t first_it, uint32_t count) {
     constexpr int UPR = G / 8;                           // 16-byte units per row of one group
     const uint32_t per_slot = (uint32_t)p.m_pad * UPR;
-    for (uint32_t q = tid; q < count * per_slot; q += 256) {
+    for (uint32_t q = tid; q < count * per_slot; q += NCONS) {
       const uint32_t k = q / per_slot, rem = q - k * per_slot;
       const uint32_t r = rem / UPR, u = rem % UPR;
       const uint32_t Gi = (g_first + first_it + k) % Gn;
@@ -185,7 +188,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qlinear_mma_kernel(const __gri
       cp_async16(xbuf + (size_t)k * xslot + r * (2 * G) + ((u ^ ((r & 1) << 2)) * 16), src, live ? 16u : 0u);
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
-    named_bar_sync(1, 256);
+    named_bar_sync(1, NCONS);
   };
   if (XP == 0) load_x_slots(0, min(my_chunks, Gn));
   float acc[4][MT][4];
@@ -204,10 +207,10 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qlinear_mma_kernel(const __gri
 
     for (uint32_t ci = 0; ci < nch; ++ci, ++it) {
       if (XP != 0 && it % XP == 0) {
-        named_bar_sync(1, 256);                          // every consumer is done with the previous phase's X
+        named_bar_sync(1, NCONS);                          // every consumer is done with the previous phase's X
         load_x_slots(it, min(XP, my_chunks - it));
       }
-      if ((int)(it & 1) != kg) continue;
+      if ((int)(it % KG) != kg) continue;
       const int s = it % NS;
       mbar_wait(&full[s], (it / NS) & 1, s_abort, p.ws.status);
       uint32_t xk;
@@ -217,34 +220,36 @@ __global__ void __launch_bounds__(kMmaThreads, 1) qlinear_mma_kernel(const __gri
         xk = g0 + ci + Gn - g_first;
         if (xk >= Gn) xk -= Gn;
       }
-      compute_chunk<MT, G>(ring + (size_t)s * stage, xbuf + (size_t)xk * xslot, wn, g8, t, acc);
+      if (!(p.ablate & 1)) compute_chunk<MT, G>(ring + (size_t)s * stage, xbuf + (size_t)xk * xslot, wn, g8, t, acc);
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[s]);
     }
 
-    // ---- end of a tile segment: add the two k-groups (fixed order: kg0 + kg1) -------------
-    if (kg == 1) {
+    // ---- end of a tile segment: add the k-groups (fixed order: kg0 + kg1 + ...) -------------
+    if (kg != 0) {
 #pragma unroll
       for (int j = 0; j < 4; ++j)
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
-          red4[((wn * 4 + j) * MT + mt) * 32 + lane] = make_float4(acc[j][mt][0], acc[j][mt][1], acc[j][mt][2], acc[j][mt][3]);
+          red4[(((kg - 1) * 16 + wn * 4 + j) * MT + mt) * 32 + lane] = make_float4(acc[j][mt][0], acc[j][mt][1], acc[j][mt][2], acc[j][mt][3]);
     }
-    named_bar_sync(1, 256);
+    named_bar_sync(1, NCONS);
     if (kg == 0) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j)
+      for (int k2 = 0; k2 < KG - 1; ++k2)
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
-          const float4 v = red4[((wn * 4 + j) * MT + mt) * 32 + lane];
-          acc[j][mt][0] += v.x; acc[j][mt][1] += v.y; acc[j][mt][2] += v.z; acc[j][mt][3] += v.w;
-        }
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            const float4 v = red4[((k2 * 16 + wn * 4 + j) * MT + mt) * 32 + lane];
+            acc[j][mt][0] += v.x; acc[j][mt][1] += v.y; acc[j][mt][2] += v.z; acc[j][mt][3] += v.w;
+          }
     }
-    named_bar_sync(1, 256);
+    named_bar_sync(1, NCONS);
     const bool whole = (g0 == 0 && nch == Gn);
     pos += nch;
     const int my_seg = seg++;
-    if (kg == 1) continue;
+    if (kg != 0) continue;
 
     // ---- k-group 0 (128 threads) finishes the segment ------------------------------------
     if (!whole) {
@@ -370,7 +375,7 @@ static cudaError_t launch_one(const LinearParams& p, size_t smem, cudaStream_t s
     if (e != cudaSuccess) return e;
     attr_set[dev] = true;
   }
-  qlinear_mma_kernel<MT, G><<<p.ncta, kMmaThreads, smem, stream>>>(p);
+  qlinear_mma_kernel<MT, G><<<p.ncta, mma_kgroups(MT) * 128 + 32, smem, stream>>>(p);
   return cudaGetLastError();
 }
 

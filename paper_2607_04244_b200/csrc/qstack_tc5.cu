@@ -664,6 +664,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
 
       // -------- chunks of this operation --------
       uint32_t pos = start, e_seg_end = 0;              // sub-chunks of the operation up to the end of the current segment
+      int am_tiles = 0;                                  // tiles of this operation the CTA has finished (arg-max bookkeeping)
       while (pos < end) {
         const uint32_t T = pos / Gn;
         const uint32_t g0 = pos - T * Gn;
@@ -834,14 +835,21 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
               const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
               st_amax_merge(bv, bi, ov, oi);
             }
-            // the warp that stores the row's last candidate reduces the candidates of all tiles
+            // Every finished tile leaves the row's candidate; the row's counter is raised once per
+            // CTA, by the number of tiles it finished, at its last tile of the operation (the last
+            // segment of a run always finishes its tile: atomics on one line from every tile of a
+            // 150,000-column head cost more than the tiles).  The warp whose addition completes
+            // the count reduces the candidates of all tiles.
             int is_last = 0;
+            ++am_tiles;
             if (lane == 0) {
               __stcg(&sp.ws.cand[(size_t)T * MP + rw], make_float2(bv, __int_as_float(bi)));
-              int old;
-              asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(sp.ws.status + 16 + rw) : "memory");
-              is_last = (old == h.n_tiles - 1);
-              if (is_last) sp.ws.status[16 + rw] = 0;
+              if (pos == end) {
+                int old;
+                asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], %2;" : "=r"(old) : "l"(sp.ws.status + 16 + rw), "r"(am_tiles) : "memory");
+                is_last = (old + am_tiles == h.n_tiles);
+                if (is_last) sp.ws.status[16 + rw] = 0;
+              }
             }
             is_last = __shfl_sync(0xffffffffu, is_last, 0);
             if (is_last && live) {
