@@ -34,9 +34,9 @@ import qsynth  # noqa: E402
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from an ncu capture of a 3-layer launch of the stack kernel:
-# dram read + write = 161.78 MB for 162.32 MB of algorithmic bytes.  Traffic grows in proportion to the
+# dram read + write = 160.79 MB for 162.32 MB of algorithmic bytes.  Traffic grows in proportion to the
 # layers streamed (every packed byte crosses HBM once), so a full launch is scaled by this ratio.
-NCU_TRAFFIC_RATIO = 161.78 / 162.32
+NCU_TRAFFIC_RATIO = 160.79 / 162.32
 
 
 # ------------------------------------------------------------------------------------------------
@@ -519,7 +519,7 @@ def run_sweep(args):
     import torch
     import paper_2607_04244_b200 as ql
     ql.load()
-    reps = 24     # distinct weight buffers per point: 24 x >= 8 MB > 2 x L2
+    reps = 36     # distinct weight buffers per point (as in the default bench line): 36 x >= 8 MB > 2 x L2
     for si, (K, N) in enumerate(qsynth.SWEEP_SHAPES):
         for g in (128, 64):
             for sym in (False, True):

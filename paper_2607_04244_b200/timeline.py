@@ -1,11 +1,16 @@
 """Per-phase timeline of the persistent stack kernel on the benchmark's verify step.
 
     python -m paper_2607_04244_b200.timeline [--layers N] [--no-lm-head]
+    python -m paper_2607_04244_b200.timeline --ablation-table
 
 Builds the instrumented twin of the library (-DQL_TIMELINE: thread 0 of every thread block stamps
 the phases of every fused operation with globaltimer), runs the benchmark step a few times and
 prints, per kind of operation, where the time of one recorded step went.  The stamps cost a few
 stores per operation; the regular library has none of them.
+
+--ablation-table uses the regular library instead: it times the step with CUDA events while parts
+of the kernel are switched off one at a time (the kernel's ablation switches; the outputs are then
+garbage and are not looked at), which shows what each part costs without any stamp in the way.
 """
 from __future__ import annotations
 
@@ -30,13 +35,63 @@ def max_pos(v, present):
     return float(v.max()) if v.size else float("nan")
 
 
+ABLATIONS = (
+    (0, "complete kernel"),
+    (16, "rows published without the release fence"),
+    (256, "watcher without its acquire fence"),
+    (64, "no row epilogue (rows are published, nothing is stored)"),
+    (32, "no accumulator exchange between the unpack groups"),
+    (8, "split tiles not exchanged between thread blocks"),
+    (2, "X operand not loaded or converted"),
+    (2 | 4, "same, and the row scales 1/rms not awaited"),
+    (1, "no weight copies, no unpacking, no MMAs"),
+    (1 | 2 | 4, "no chunks, no X"),
+    (1 | 2 | 4 | 8 | 32 | 64, "synchronisation skeleton only (dependency waits, barriers, publishing)"),
+)
+
+
+def ablation_table(args):
+    import torch
+    import paper_2607_04244_b200 as ql
+    ql.load()
+    import bench
+    step = bench.VerifyStep(ql, torch, 16, 128, n_layers=args.layers, lm_head=not args.no_lm_head)
+    n_ops = 4 * args.layers + (0 if args.no_lm_head else 1)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rows = []
+    for mask, what in ABLATIONS:
+        ql.ql_debug_set_ablate(mask)
+        for _ in range(3):
+            step.run()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(args.steps):
+            step.run()
+        e1.record()
+        torch.cuda.synchronize()
+        rows.append((mask, what, e0.elapsed_time(e1) / args.steps))
+    ql.ql_debug_set_ablate(0)
+    step.run()
+    torch.cuda.synchronize()
+    assert ql.ql_device_status(step.ws) == ql.QL_OK
+    full = rows[0][2]
+    print(f"{n_ops} fused operations per step, {args.steps} steps per row, CUDA events")
+    print(f"{'mask':>5s}  {'ms/step':>8s}  {'saved':>7s}  {'us/op':>6s}  what is switched off")
+    for mask, what, ms in rows:
+        print(f"{mask:5d}  {ms:8.3f}  {full - ms:7.3f}  {ms * 1e3 / n_ops:6.2f}  {what}")
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--ablation-table", action="store_true", help="time the step with parts of the kernel switched off (regular library)")
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--layers", type=int, default=36)
     ap.add_argument("--no-lm-head", action="store_true")
     ap.add_argument("--ablate", type=int, default=0, help="ablation mask of the stack kernel (timing experiments)")
     ap.add_argument("--json", default=None, help="also write the per-kind medians to this file")
     args = ap.parse_args()
+    if args.ablation_table:
+        return ablation_table(args)
     import torch
     from paper_2607_04244_b200 import build
     import paper_2607_04244_b200 as ql
