@@ -273,6 +273,40 @@ int qlinear_w4a16_static(const void* packed, const uint16_t* X, uint16_t* Y, int
                          int M, int K, int N, int g, void* stream);
 int ql_static_status(int* host_out, void* stream);
 
+/* Symmetric sliding-window attention of a drafted block (paper Section 3.3, "Drafter SWA": the
+ * drafter's mask-token queries attend bidirectionally, each restricted to a fixed-size window that
+ * is symmetric around the query; the window is applied inside the attention computation only, the
+ * key/value cache stays complete; sequences that fit into the window are attended in full.
+ * Section 2.3 for why the drafter has it).
+ *
+ *   query i (0 <= i < n_q) stands at position p0 + i and sees the keys k with
+ *   |k - (p0 + i)| <= window / 2 (integer division), clipped to [0, T); every key if T <= window.
+ *   out[i, h, :] = sum_k softmax_k(Q[i,h,:] . K[k, h / (Hq/Hkv), :] / sqrt(d)) * V[k, h / (Hq/Hkv), :]
+ *   over the visible keys; bf16 in and out, fp32 arithmetic (probabilities enter the second
+ *   contraction with 16 significant bits).
+ *
+ *   Q    DEVICE, bf16 [n_q][Hq][d], ld_q elements between consecutive queries (>= Hq*d)
+ *   K, V DEVICE, bf16 [T][Hkv][d], ld_kv elements between consecutive positions (>= Hkv*d):
+ *        the complete cache; positional rotation, if any, has been applied before
+ *   out  DEVICE, bf16 [n_q][Hq][d], ld_out elements between consecutive queries
+ *   1 <= n_q <= 16, d == 128, Hq/Hkv in {1, 2, 4, 8}, 0 <= p0, p0 + n_q <= T, window >= 0;
+ *   leading dimensions multiples of 8, pointers 16-byte aligned
+ *   workspace DEVICE, >= ql_attn_workspace_bytes(Hq, Hkv) bytes, zeroed once with ql_workspace_init
+ *        (it is NOT the workspace of the linear calls: the two may not share memory that is in use
+ *        at the same time); holds the partial rows of the key pieces and one counter per head
+ *
+ * Asynchronous on `stream`, no allocation, no host synchronisation; nothing in the kernel waits for
+ * another thread block.  Results are bit-identical from run to run.  Errors as the other calls
+ * (QL_ERR_SHAPE for positions outside the cache, QL_ERR_UNSUPPORTED for other head sizes).
+ * ql_attn_plan reports what a call would do: out = {first visible key, one past the last, key
+ * pieces per head, 64-key sub-blocks per piece}; it needs no device.
+ */
+size_t ql_attn_workspace_bytes(int Hq, int Hkv);
+int qattn_swa_bf16(const uint16_t* Q, const uint16_t* K, const uint16_t* V, uint16_t* out,
+                   int n_q, int T, int Hq, int Hkv, int d, int p0, int window,
+                   int ld_q, int ld_kv, int ld_out, void* workspace, size_t workspace_bytes, void* stream);
+int ql_attn_plan(int n_q, int T, int Hq, int Hkv, int d, int p0, int window, int out[4]);
+
 /* The stream-K split the persistent kernels use (host copies of the device arithmetic, for tests):
  * the first min(ncta, total_chunks) CTAs share an operation's chunks, CTA i owning
  * [ql_plan_first_chunk(.., i), ql_plan_first_chunk(.., i+1)); ql_plan_chunk_owner is the inverse. */

@@ -24,6 +24,7 @@ EXPORTS = [
     "ql_device_status_raw",
     "qpack_w4_g128", "qrequant_pack_w4", "qlinear_w4a16", "qlinear_w4a16_path", "ql_select_path", "qlinear_stack_w4a16",
     "qlinear_stack_w4a16_host", "ql_launch_count", "qlinear_w4a16_static", "ql_static_status", "ql_stack_plan", "ql_linear_plan", "ql_plan_first_chunk", "ql_plan_chunk_owner",
+    "ql_attn_workspace_bytes", "qattn_swa_bf16", "ql_attn_plan",
     "ql_debug_set_wait_budget_ns", "ql_debug_no_release", "ql_debug_set_timeline", "ql_debug_timeline_enabled", "ql_debug_set_ablate",
 ]
 
@@ -93,6 +94,12 @@ def load(path: str | None = None):
     lib.ql_stack_plan.argtypes = [ctypes.POINTER(ql_op), i32, vp, sz, ctypes.POINTER(ctypes.c_int)]
     lib.ql_linear_plan.restype = i32
     lib.ql_linear_plan.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(ctypes.c_int)]
+    lib.ql_attn_workspace_bytes.restype = sz
+    lib.ql_attn_workspace_bytes.argtypes = [i32, i32]
+    lib.qattn_swa_bf16.restype = i32
+    lib.qattn_swa_bf16.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, i32, vp, sz, vp]
+    lib.ql_attn_plan.restype = i32
+    lib.ql_attn_plan.argtypes = [i32, i32, i32, i32, i32, i32, i32, ctypes.POINTER(ctypes.c_int)]
     for fn in (lib.ql_plan_first_chunk, lib.ql_plan_chunk_owner):
         fn.restype = ctypes.c_uint32
         fn.argtypes = [ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32]
@@ -267,6 +274,38 @@ def ql_static_status(stream=None) -> int:
     out = ctypes.c_int(-1)
     _check(load().ql_static_status(ctypes.byref(out), _stream(stream)), "ql_static_status")
     return out.value
+
+
+def ql_attn_workspace_bytes(Hq: int, Hkv: int) -> int:
+    return int(load().ql_attn_workspace_bytes(Hq, Hkv))
+
+
+def new_attn_workspace(Hq: int, Hkv: int, device="cuda", stream=None):
+    """Allocate (with torch) and zero a workspace for qattn_swa_bf16."""
+    import torch
+    nbytes = ql_attn_workspace_bytes(Hq, Hkv)
+    if nbytes == 0:
+        raise QlError(QL_ERR_SHAPE, "ql_attn_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    ql_workspace_init(ws, stream)
+    return ws
+
+
+def qattn_swa_bf16(Q, K, V, out, n_q: int, T: int, Hq: int, Hkv: int, d: int, p0: int, window: int, ws,
+                   ld_q=None, ld_kv=None, ld_out=None, stream=None):
+    """Q int16 (bf16 bits) [n_q,Hq,d], K / V [T,Hkv,d], out [n_q,Hq,d]; leading dimensions default to dense."""
+    _check(load().qattn_swa_bf16(Q.data_ptr(), K.data_ptr(), V.data_ptr(), out.data_ptr(), n_q, T, Hq, Hkv, d, p0, window,
+                                 Hq * d if ld_q is None else ld_q, Hkv * d if ld_kv is None else ld_kv,
+                                 Hq * d if ld_out is None else ld_out, ws.data_ptr(), ws.numel(), _stream(stream)),
+           "qattn_swa_bf16")
+    return out
+
+
+def ql_attn_plan(n_q: int, T: int, Hq: int, Hkv: int, d: int, p0: int, window: int) -> dict:
+    """What qattn_swa_bf16 would do (no launch, no device needed)."""
+    c = (ctypes.c_int * 4)()
+    _check(load().ql_attn_plan(n_q, T, Hq, Hkv, d, p0, window, c), "ql_attn_plan")
+    return dict(zip(["key_lo", "key_hi", "n_pieces", "sub_per_piece"], list(c)))
 
 
 def ql_linear_plan(M: int, K: int, N: int, g: int, path: int = QL_PATH_AUTO) -> dict:

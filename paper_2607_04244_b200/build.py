@@ -9,7 +9,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libqlinear_w4a16.so")
 LIB_PATH_TIMELINE = os.path.join(PKG_DIR, "libqlinear_w4a16_timeline.so")   # same library built with -DQL_TIMELINE
-SOURCES = ["api.cu", "qpack.cu", "glue.cu", "qlinear_mma.cu", "qlinear_tc5.cu", "qstack_tc5.cu", "qlinear_static.cu"]
+SOURCES = ["api.cu", "qpack.cu", "glue.cu", "qlinear_mma.cu", "qlinear_tc5.cu", "qstack_tc5.cu", "qlinear_static.cu", "qattn_swa.cu"]
 HEADERS = ["ql_device.cuh", "ql_params.h", os.path.join("..", "..", "include", "qlinear_w4a16.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--shared", "-Xcompiler", "-fPIC"]

@@ -11,6 +11,8 @@ namespace ql {
 cudaError_t launch_qpack(const uint32_t*, const uint16_t*, const uint8_t*, int, int, int, uint8_t*, cudaStream_t);
 cudaError_t launch_qrequant(const uint16_t*, const uint16_t*, const uint8_t*, int, int, int, uint8_t*, cudaStream_t);
 cudaError_t launch_linear_mma(LinearParams, cudaStream_t);
+size_t attn_plan(AttnParams&, int sms);
+cudaError_t launch_attn_swa(const AttnParams&, cudaStream_t);
 size_t plan_linear_mma(LinearParams&);
 cudaError_t launch_linear_tc5(LinearParams, int sms, cudaStream_t, bool pdl);
 bool tc5_supported(const LinearParams&, int sms);
@@ -480,6 +482,65 @@ int qrequant_pack_w4(const uint16_t* w, const uint16_t* scale, const uint8_t* ze
   if (launch_qrequant(w, scale, zero, K, N, g, static_cast<uint8_t*>(packed), static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return QL_ERR_CUDA;
   g_launches.fetch_add(1, std::memory_order_relaxed);
+  return QL_OK;
+}
+
+// ---- drafter attention ----------------------------------------------------------------------
+constexpr size_t kAttnCounterBytes = 256;                // one counter per key/value head, zero between calls
+
+static int attn_fill(AttnParams& p, int n_q, int T, int Hq, int Hkv, int d, int p0, int window, int ld_q, int ld_kv, int ld_out) {
+  if (d != 128) return QL_ERR_UNSUPPORTED;
+  if (n_q < 1 || n_q > 16 || T < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || Hkv > 64 || window < 0) return QL_ERR_SHAPE;
+  const int G = Hq / Hkv;
+  if (G != 1 && G != 2 && G != 4 && G != 8) return QL_ERR_UNSUPPORTED;
+  if (p0 < 0 || p0 + n_q > T) return QL_ERR_SHAPE;        // every query stands on a position of the cache
+  if (ld_q < Hq * d || ld_out < Hq * d || ld_kv < Hkv * d) return QL_ERR_SHAPE;
+  if (ld_q % 8 != 0 || ld_kv % 8 != 0 || ld_out % 8 != 0) return QL_ERR_ALIGN;
+  p.n_q = n_q; p.T = T; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.p0 = p0; p.window = window;
+  p.ld_q = ld_q; p.ld_kv = ld_kv; p.ld_out = ld_out;
+  p.scale_log2 = 1.4426950408889634f / sqrtf((float)d);
+  return QL_OK;
+}
+
+size_t ql_attn_workspace_bytes(int Hq, int Hkv) {
+  if (Hq < 1 || Hkv < 1 || Hq % Hkv != 0) return 0;
+  int sms = num_sms();
+  if (sms <= 0) sms = 148;                              // no device: answer for a B200
+  int pieces = sms / Hkv;
+  if (pieces < 1) pieces = 1;
+  const size_t need = kAttnCounterBytes + (size_t)Hq * pieces * 16 * 132 * sizeof(float);
+  return need < kWsControlBytes ? kWsControlBytes : need;   // ql_workspace_init zeroes it: not smaller than what that call accepts
+}
+
+int qattn_swa_bf16(const uint16_t* Q, const uint16_t* K, const uint16_t* V, uint16_t* out, int n_q, int T, int Hq, int Hkv,
+                   int d, int p0, int window, int ld_q, int ld_kv, int ld_out, void* workspace, size_t workspace_bytes,
+                   void* stream) {
+  if (Q == nullptr || K == nullptr || V == nullptr || out == nullptr || workspace == nullptr) return QL_ERR_NULL;
+  AttnParams p = {};
+  const int st = attn_fill(p, n_q, T, Hq, Hkv, d, p0, window, ld_q, ld_kv, ld_out);
+  if (st != QL_OK) return st;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(out) || !aligned16(workspace)) return QL_ERR_ALIGN;
+  const int sms = num_sms();
+  if (sms <= 0) return QL_ERR_CUDA;
+  const size_t floats = attn_plan(p, sms);
+  if (workspace_bytes < kAttnCounterBytes + floats * sizeof(float)) return QL_ERR_WORKSPACE;
+  p.Q = Q; p.K = K; p.V = V; p.out = out;
+  p.counters = static_cast<int*>(workspace);
+  p.part = reinterpret_cast<float*>(static_cast<char*>(workspace) + kAttnCounterBytes);
+  if (launch_attn_swa(p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return QL_ERR_CUDA;
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return QL_OK;
+}
+
+int ql_attn_plan(int n_q, int T, int Hq, int Hkv, int d, int p0, int window, int out[4]) {
+  if (out == nullptr) return QL_ERR_NULL;
+  AttnParams p = {};
+  const int st = attn_fill(p, n_q, T, Hq, Hkv, d, p0, window, Hq * d, Hkv * d, Hq * d);
+  if (st != QL_OK) return st;
+  int sms = num_sms();
+  if (sms <= 0) sms = 148;                              // no device: answer for a B200
+  attn_plan(p, sms);
+  out[0] = p.key_lo; out[1] = p.key_hi; out[2] = p.n_pieces; out[3] = p.sub_per_piece;
   return QL_OK;
 }
 

@@ -119,4 +119,20 @@ __host__ __device__ inline uint32_t chunk_owner(uint32_t c, uint32_t total, uint
   return (uint32_t)((((uint64_t)c + 1) * ncta + total - 1) / total) - 1;
 }
 
+// Sliding-window attention of a drafted block (qattn_swa.cu).
+struct AttnParams {
+  const uint16_t* Q;
+  const uint16_t* K;
+  const uint16_t* V;
+  uint16_t* out;
+  float* part;            // [Hkv][n_pieces][G][16][kAttnPartStride]
+  int* counters;          // [Hkv], zero between calls
+  int n_q, T, Hq, Hkv, G;
+  int p0, window;
+  int ld_q, ld_kv, ld_out;   // elements between consecutive queries / tokens / output rows
+  int key_lo, key_hi;        // union of the visible keys of all queries
+  int sub_per_piece, n_pieces;
+  float scale_log2;          // log2(e) / sqrt(d)
+};
+
 }  // namespace ql

@@ -21,7 +21,6 @@
 
 namespace ql {
 
-constexpr int kMmaMaxThreads = 544;                     // 4 k-groups of 4 warps + the producer warp
 __host__ __device__ constexpr int mma_kgroups(int mt) { return mt == 1 ? 4 : 2; }   // k-groups (sets of 4 consumer warps taking alternate chunks)
 constexpr int kMaxStages = 32;
 constexpr uint32_t kSmemBudget = 232448u;   // 227 KB of dynamic shared memory per CTA

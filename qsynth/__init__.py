@@ -148,3 +148,20 @@ def config4_point(shape_idx: int, M: int, g: int, symmetric: bool) -> dict:
     d["x"] = make_x([4, shape_idx, g, int(symmetric), M], M, K)
     d["M"] = M
     return d
+
+
+# --------------------------------------------------------------------------------------------
+# drafter attention (synthetic stand-ins for the drafter's queries and its key/value cache)
+
+ATTN_HEADS, ATTN_KV_HEADS, ATTN_HEAD_DIM = 32, 8, 128     # the target's synthetic geometry (4096 = 32 x 128, 1024 = 8 x 128)
+SWA_CONTEXTS = (64, 2048, 8192)                          # input lengths of the paper's three latency settings
+SWA_WINDOWS = (1024, 2048)
+
+
+def attention_inputs(entropy, n_q: int, T: int, Hq: int, Hkv: int, d: int = ATTN_HEAD_DIM):
+    """bf16 bit patterns: q [n_q, Hq, d], k and v [T, Hkv, d], all N(0,1); draw order q, k, v."""
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([0x5A, int(entropy)])))
+    q = f32_to_bf16_bits(rng.standard_normal((n_q, Hq, d), dtype=np.float32))
+    k = f32_to_bf16_bits(rng.standard_normal((T, Hkv, d), dtype=np.float32))
+    v = f32_to_bf16_bits(rng.standard_normal((T, Hkv, d), dtype=np.float32))
+    return q, k, v

@@ -55,6 +55,26 @@ def test_size_queries(pkg):
     assert pkg.ql_select_path(16, 2560, 9728, 96) < 0
 
 
+def test_attention_plan_and_argument_checks_without_a_device(pkg):
+    # the union of the queries' windows and its split into pieces of 64-key sub-blocks (paper Section 3.3)
+    assert pkg.ql_attn_plan(16, 8208, 32, 8, 128, 8192, 1024) == dict(key_lo=8192 - 512, key_hi=8208, n_pieces=9, sub_per_piece=1)
+    assert pkg.ql_attn_plan(16, 2064, 32, 8, 128, 2048, 2048) == dict(key_lo=1024, key_hi=2064, n_pieces=17, sub_per_piece=1)
+    assert pkg.ql_attn_plan(16, 80, 32, 8, 128, 64, 1024) == dict(key_lo=0, key_hi=80, n_pieces=2, sub_per_piece=1)      # fits: everything
+    p = pkg.ql_attn_plan(16, 4096, 32, 8, 128, 2000, 1024)
+    assert (p["key_lo"], p["key_hi"]) == (1488, 2528)                                   # both sides of the block
+    p = pkg.ql_attn_plan(16, 40016, 32, 8, 128, 40000, 65536)
+    assert p["n_pieces"] * p["sub_per_piece"] * 64 >= 40016 and p["n_pieces"] <= 18
+    for bad in [(17, 100, 32, 8, 128, 0, 64), (16, 100, 32, 8, 128, 90, 64), (16, 100, 32, 5, 128, 0, 64), (0, 100, 32, 8, 128, 0, 64)]:
+        with pytest.raises(pkg.QlError) as e:
+            pkg.ql_attn_plan(*bad)
+        assert e.value.status == pkg.QL_ERR_SHAPE
+    with pytest.raises(pkg.QlError) as e:
+        pkg.ql_attn_plan(16, 100, 32, 8, 64, 0, 64)
+    assert e.value.status == pkg.QL_ERR_UNSUPPORTED
+    assert pkg.ql_attn_workspace_bytes(32, 8) >= 256 + 32 * 18 * 16 * 132 * 4
+    assert pkg.ql_attn_workspace_bytes(32, 5) == 0
+
+
 def test_status_strings(pkg):
     lib = pkg.load()
     seen = {lib.ql_status_str(i).decode() for i in range(8)}
