@@ -13,6 +13,7 @@ N > 1 (under torchrun): every rank runs an independent replica of the step on it
 (the path has no exchange step); value is the aggregate over ranks, time is the max over ranks.
 --impl reference times the CPU oracle on a bounded sample of the same workload.
 --sweep prints one JSON line per point of the M-sweep (M x shape x group size x zero mode).
+--swa prints the drafter's sliding-window attention points only.
 """
 from __future__ import annotations
 
@@ -214,6 +215,52 @@ def independent_point(ql, torch, M, K, N, g, packed, ws, sym=False, iters=5):
     return {"M": M, "K": K, "N": N, "g": g, "zero": "sym8" if sym else "asym", "us": us, "us_min": ts[0], "bytes": b,
             "GBps": b / us / 1e3, "frac_of_measured_peak": b / us / 1e3 / peak, "frac_of_8TBs": b / us / 1e3 / NOMINAL_HBM_GBS,
             "kernel": kernel, "weight_sets": R}
+
+
+def swa_points(ql, torch, caches=32, iters=5):
+    """The drafter's sliding-window attention (paper Section 3.3) at the paper's three input lengths and its
+    two windows, plus full attention at the long length: `caches` distinct key/value caches back to
+    back (together more than twice the L2 wherever a call reads more than a few MB), one call each,
+    time / caches.  Bytes = the keys and values inside the union of the 16 queries' windows + Q + out."""
+    Hq, Hkv, d, n_q = qsynth.ATTN_HEADS, qsynth.ATTN_KV_HEADS, qsynth.ATTN_HEAD_DIM, 16
+    ws = ql.new_attn_workspace(Hq, Hkv)
+    peak, _ = measured_peak()
+    rows = []
+    for ctx in qsynth.SWA_CONTEXTS:
+        T = ctx + n_q
+        K = [torch.randn((T, Hkv * d), device="cuda").to(torch.bfloat16).view(torch.int16) for _ in range(caches)]
+        V = [torch.randn((T, Hkv * d), device="cuda").to(torch.bfloat16).view(torch.int16) for _ in range(caches)]
+        Q = torch.randn((n_q, Hq * d), device="cuda").to(torch.bfloat16).view(torch.int16)
+        outs = [torch.zeros((n_q, Hq * d), dtype=torch.int16, device="cuda") for _ in range(caches)]
+        for window in qsynth.SWA_WINDOWS + ((1 << 20,) if ctx == qsynth.SWA_CONTEXTS[-1] else ()):
+            plan = ql.ql_attn_plan(n_q, T, Hq, Hkv, d, ctx, window)
+
+            def fn():
+                for k, v, o in zip(K, V, outs):
+                    ql.qattn_swa_bf16(Q, k, v, o, n_q, T, Hq, Hkv, d, ctx, window, ws)
+            for _ in range(2):
+                fn()
+            torch.cuda.synchronize()
+            # a call takes less device time than the host needs to enqueue it through the binding: the
+            # stream is held back by a spin kernel while the calls are enqueued, so that the events
+            # bracket device time only
+            def timed():
+                a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda._sleep(6_000_000)
+                a.record()
+                fn()
+                e.record()
+                e.synchronize()
+                return a.elapsed_time(e)
+            ts = sorted(timed() / caches * 1e3 for _ in range(iters))
+            us = ts[len(ts) // 2]
+            b = 2 * (plan["key_hi"] - plan["key_lo"]) * Hkv * d * 2 + 2 * n_q * Hq * d * 2
+            rows.append({"context": ctx, "window": "full" if window >= T else window, "keys_read": plan["key_hi"] - plan["key_lo"],
+                         "thread_blocks": plan["n_pieces"] * Hkv, "us": us, "us_min": ts[0], "bytes": b, "GBps": b / us / 1e3,
+                         "frac_of_measured_peak": b / us / 1e3 / peak, "kernel": "qattn_swa_kernel, one launch per call"})
+        del K, V, outs
+        torch.cuda.empty_cache()
+    return rows
 
 
 def max_over_ranks(x: float, world: int, device="cuda") -> float:
@@ -453,6 +500,8 @@ def run_ours(args, rank, world, local_rank):
         lm_point = {"us": ts[len(ts) // 2], "us_min": ts[0], "bytes": b, "GBps": b / ts[len(ts) // 2] / 1e3,
                     "frac_of_measured_peak": b / ts[len(ts) // 2] / 1e3 / peak, "kernel": "qstack_tc5_kernel (tokens only, no Y)"}
 
+    swa_block = swa_points(ql, torch) if (rank == 0 and not args.no_extras) else None
+
     if rank != 0:
         return
     line = {"metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
@@ -467,7 +516,7 @@ def run_ours(args, rank, world, local_rank):
             "e2e": {"value": e2e_val, "unit": "GB/s", "h2d_bytes_per_step": int(step.host_in.numel() * 2),
                     "d2h_bytes_per_step": int(step.host_tokens.numel() * 4), "ms_per_step": e2e_s * 1e3},
             "roofline": roofline, "single_linear_cold_l2_m16": extras, "lm_head_m16": lm_point, "m_sweep": sweep_block,
-            "tokens_agree_device_vs_host_entry": tokens_agree}
+            "drafter_swa_attention": swa_block, "tokens_agree_device_vs_host_entry": tokens_agree}
     if world == 1 and not args.no_cpu_baseline:
         sec, n_sample = oracle_sample_seconds(12, M, g)
         line["cpu_baseline"] = {"value": per_layer * n_sample / sec / 1e9, "unit": "GB/s", "cores": host_threads(),
@@ -599,6 +648,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--swa", action="store_true", help="only the drafter's sliding-window attention points, one JSON line")
     ap.add_argument("--workload", default="verify_step", choices=["verify_step", "drafter"],
                     help="drafter: the second workload (5 symmetric-INT4 layers, synthetic widths)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -618,6 +668,12 @@ def main():
         return
     if args.workload == "drafter":
         run_drafter(args)
+        return
+    if args.swa:
+        import torch
+        import paper_2607_04244_b200 as ql
+        ql.load()
+        print(json.dumps({"drafter_swa_attention": swa_points(ql, torch), "gpu_launches": int(ql.ql_launch_count())}), flush=True)
         return
     if args.sweep:
         run_sweep(args)

@@ -59,7 +59,7 @@ def test_attention_plan_and_argument_checks_without_a_device(pkg):
     # the union of the queries' windows and its split into pieces of 64-key sub-blocks (paper Section 3.3)
     assert pkg.ql_attn_plan(16, 8208, 32, 8, 128, 8192, 1024) == dict(key_lo=8192 - 512, key_hi=8208, n_pieces=9, sub_per_piece=1)
     assert pkg.ql_attn_plan(16, 2064, 32, 8, 128, 2048, 2048) == dict(key_lo=1024, key_hi=2064, n_pieces=17, sub_per_piece=1)
-    assert pkg.ql_attn_plan(16, 80, 32, 8, 128, 64, 1024) == dict(key_lo=0, key_hi=80, n_pieces=2, sub_per_piece=1)      # fits: everything
+    assert pkg.ql_attn_plan(16, 80, 32, 8, 128, 64, 1024) == dict(key_lo=0, key_hi=80, n_pieces=1, sub_per_piece=2)      # fits: everything, one piece
     p = pkg.ql_attn_plan(16, 4096, 32, 8, 128, 2000, 1024)
     assert (p["key_lo"], p["key_hi"]) == (1488, 2528)                                   # both sides of the block
     p = pkg.ql_attn_plan(16, 40016, 32, 8, 128, 40000, 65536)
