@@ -183,6 +183,36 @@ def test_independent_linears_in_one_stack_call(ql):
     check_against_oracle(host_u16(ytail), y64, "dependent tail")
 
 
+def test_dependency_at_distance_three_over_small_operations(ql):
+    """A large linear, two small independent ones that most thread blocks have no chunk of, then
+    a linear that reads the first one's output: a thread block that skipped the small operations
+    must still not read that output before every tile of it is finished."""
+    M, g = 16, 128
+    A = qsynth.make_linear([97, 0], M, 2560, 1024, g)          # 160 chunks: every thread block takes part
+    B = qsynth.make_linear([97, 1], M, 1024, 1024, g)          # 64 chunks: fewer than thread blocks
+    C = qsynth.make_linear([97, 2], M, 1024, 1024, g)
+    D = qsynth.make_linear([97, 3], M, 1024, 2560, g)          # reads A's output
+    pk = [pack_on_device(ql, d) for d in (A, B, C, D)]
+    xa, xb, xc = dev_u16(A["x"]), dev_u16(B["x"]), dev_u16(C["x"])
+    ya, yb, yc = (torch.full((M, 1024), 0x7FC0, dtype=torch.int16, device="cuda") for _ in range(3))
+    yd = torch.full((M, 2560), 0x7FC0, dtype=torch.int16, device="cuda")
+    lin = lambda d, p, x, y: dict(kind=ql.QL_OP_LINEAR, M=M, K=d["K"], N=d["N"], g=g, ld_in=d["K"], ld_out=d["N"], packed=p, in0=x, out=y)
+    arr = ql.make_ops([lin(A, pk[0], xa, ya), lin(B, pk[1], xb, yb), lin(C, pk[2], xc, yc), lin(D, pk[3], ya, yd)])
+    ws = ql.new_workspace(M, 2560)
+    plan = ql.ql_stack_plan(arr, ws.data_ptr(), ws.numel())
+    assert plan["stack_launches"] == 1 and plan["batch_launches"] == 0 and plan["independent"] == 0   # a chain: everybody waits
+    for rep in range(5):
+        ya.fill_(0x7FC0)
+        yd.fill_(0x7FC0)
+        ql.qlinear_stack_w4a16(arr, ws)
+        torch.cuda.synchronize()
+        assert ql.ql_device_status(ws) == ql.QL_OK
+        y64 = orc.qlinear_f64(host_u16(ya), D["wq"], D["scale"], D["zero"], g)
+        check_against_oracle(host_u16(yd), y64, f"D after A, repetition {rep}")
+    for d, y in ((A, ya), (B, yb), (C, yc)):
+        check_against_oracle(host_u16(y), orc.qlinear_f64(d["x"], d["wq"], d["scale"], d["zero"], g), "A/B/C")
+
+
 def test_full_verify_step_one_launch_sampled_layers(ql):
     """The benchmark's step at full size and in the launch configuration bench.py times: 36 layers
     + LM head with arg-max in ONE qlinear_stack_w4a16 call (one launch of the persistent kernel).
