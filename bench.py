@@ -630,7 +630,15 @@ def run_linears(args):
     ops = ql.make_ops([dict(kind=ql.QL_OP_LINEAR, M=M, K=K, N=N, g=g, ld_in=K, ld_out=N, packed=p, in0=xin, out=y)
                        for p, y in zip(packed, youts)])
     plan = ql.ql_stack_plan(ops, ws.data_ptr(), ws.numel())
-    fn = lambda: ql.qlinear_stack_w4a16(ops, ws)
+    if args.path == "stack":
+        fn = lambda: ql.qlinear_stack_w4a16(ops, ws)
+    else:
+        forced = ql.QL_PATH_MMA if args.path == "mma" else ql.QL_PATH_TC5
+
+        def fn():
+            for pk, y in zip(packed, youts):
+                ql.qlinear_w4a16(pk, xin, y, None, M, K, N, g, ws, path=forced)
+        plan = {"one launch per linear": args.path}
     for _ in range(max(args.warmup, 3)):
         fn()
     torch.cuda.synchronize()
@@ -657,6 +665,8 @@ def main():
     ap.add_argument("--no-lm-head", action="store_true", help="leave the LM head out (profiler captures)")
     ap.add_argument("--no-extras", action="store_true", help="skip the single-linear and end-to-end legs")
     ap.add_argument("--paths", action="store_true", help="forced-path comparison (mma.sync vs tcgen05), one launch per linear")
+    ap.add_argument("--path", default="stack", choices=["stack", "mma", "tcgen05"],
+                    help="with --linears: one stack call (default) or one forced-path qlinear_w4a16 launch per linear")
     ap.add_argument("--linears", default=None, metavar="K,N,R",
                     help="instead of the verify step: R independent 16xKxN linears in one call (batch kernel)")
     args = ap.parse_args()
