@@ -293,7 +293,8 @@ int ql_static_status(int* host_out, void* stream);
  *   leading dimensions multiples of 8, pointers 16-byte aligned
  *   workspace DEVICE, >= ql_attn_workspace_bytes(Hq, Hkv) bytes, zeroed once with ql_workspace_init
  *        (it is NOT the workspace of the linear calls: the two may not share memory that is in use
- *        at the same time); holds the partial rows of the key pieces and one counter per head
+ *        at the same time); holds the partial rows of the key pieces and one counter per head;
+ *        calls that may overlap on the GPU (different streams) need workspaces of their own
  *
  * Asynchronous on `stream`, no allocation, no host synchronisation; nothing in the kernel waits for
  * another thread block.  Results are bit-identical from run to run.  Errors as the other calls
