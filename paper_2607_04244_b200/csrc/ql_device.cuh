@@ -118,6 +118,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
+// The same with a suspend-time hint: a thread that finds the phase incomplete may be suspended by the
+// hardware for up to `hint_ns` (it is resumed when the phase completes), instead of spinning on
+// the instruction and taking issue slots from the warps that work.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
+
 // Bounded wait on an mbarrier phase.  Gives up after kWaitBudgetNs: records QL_ERR_DEVICE_TIMEOUT
 // in the status word, raises the CTA-wide abort flag and returns, so that every later wait of
 // the CTA falls through at once and the kernel runs to its end (with garbage results, which the

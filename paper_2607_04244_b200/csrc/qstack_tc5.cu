@@ -125,12 +125,14 @@ __device__ __forceinline__ void wait_fail(const WaitCtx& w, int site) {
   atomicCAS(w.status, 0, kStatusTimeout | (site << 8) | ((int)blockIdx.x << 16));
 }
 // Bounded wait on an mbarrier phase (see mbar_wait; the budget is a launch parameter here).
+// (SUSPEND: the single-thread roles that wait most of the time let the hardware suspend them)
+template <bool SUSPEND = false>
 __device__ __forceinline__ void st_mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtx& w, int site) {
   if (mbar_try_wait(bar, parity)) return;
   if (*w.s_abort) return;
   const uint64_t t0 = globaltimer_ns();
   uint32_t spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
+  while (!(SUSPEND ? mbar_try_wait_hint(bar, parity, 2000u) : mbar_try_wait(bar, parity))) {
     if ((++spins & 63u) == 0) {
       if (*w.s_abort) return;
       if (globaltimer_ns() - t0 > w.budget) { wait_fail(w, site); return; }
@@ -531,7 +533,10 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
           for (int hh = 0; hh < 2; ++hh, ++hs) {
             const uint32_t slot = hs % AH;
             QL_CYC_BEGIN();
-            st_mbar_wait(&a_full[w * AH + slot], (hs / AH) & 1, wc, 3);
+            // in a chain the issuer waits most of the time (for X, for the predecessor): suspended it leaves
+            // the issue slots to the unpack warps; on a stream its wake-up would cost more than its polling
+            if (h.flags & kOpWait) st_mbar_wait<true>(&a_full[w * AH + slot], (hs / AH) & 1, wc, 3);
+            else st_mbar_wait(&a_full[w * AH + slot], (hs / AH) & 1, wc, 3);
             QL_CYC_END(0);
             if (first) {
               st_mbar_wait(x_full, (xops - 1) & 1, wc, 2);   // X of this operation is in shared memory
