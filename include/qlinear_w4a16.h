@@ -196,6 +196,11 @@ int ql_linear_plan(int M, int K, int N, int g, int path, int out[4]);
  * ql_stack_plan tells what a list turns into.  The call stages the fused
  * operation descriptors from host memory into the workspace with an asynchronous copy, so it is
  * not meant to be recorded by stream capture.
+ * A call that resolves to one launch of the persistent kernel is remembered per host thread: the
+ * same call again (byte-identical operation list, same workspace, size and stream, and nothing
+ * staged into any workspace by any thread in between) skips planning and the descriptor copy and
+ * only launches.  A changed field of an operation, another list, ql_workspace_init or any
+ * ql_debug_* setter makes the next call plan again.
  * Errors: as qlinear_w4a16, reported for the first offending operation; nothing is launched
  * unless every operation validates.
  */

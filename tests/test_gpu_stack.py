@@ -213,6 +213,36 @@ def test_dependency_at_distance_three_over_small_operations(ql):
         check_against_oracle(host_u16(y), orc.qlinear_f64(d["x"], d["wq"], d["scale"], d["zero"], g), "A/B/C")
 
 
+def test_repeated_and_alternating_calls_with_one_workspace(ql):
+    """A repeated call may reuse the staged descriptors; a different list in between, a changed
+    pointer inside an otherwise equal list, or a re-initialised workspace must all be noticed."""
+    M, g = 16, 128
+    a = qsynth.make_linear([96, 0], M, 1024, 1536, g)
+    b = qsynth.make_linear([96, 1], M, 1024, 1536, g)
+    pa, pb = pack_on_device(ql, a), pack_on_device(ql, b)
+    xa, xb = dev_u16(a["x"]), dev_u16(b["x"])
+    ya, yb, yc = (torch.full((M, 1536), 0x7FC0, dtype=torch.int16, device="cuda") for _ in range(3))
+    lin = lambda d, p, x, y: ql.make_ops([dict(kind=ql.QL_OP_LINEAR, M=M, K=1024, N=1536, g=g, ld_in=1024, ld_out=1536, packed=p, in0=x, out=y)])
+    ops_a, ops_b, ops_a2 = lin(a, pa, xa, ya), lin(b, pb, xb, yb), lin(a, pa, xa, yc)
+    ws = ql.new_workspace(M, 1536)
+    want_a = orc.qlinear_f64(a["x"], a["wq"], a["scale"], a["zero"], g)
+    want_b = orc.qlinear_f64(b["x"], b["wq"], b["scale"], b["zero"], g)
+    n0 = ql.ql_launch_count()
+    for ops, y, want in ((ops_a, ya, want_a), (ops_a, ya, want_a), (ops_b, yb, want_b), (ops_a, ya, want_a), (ops_a2, yc, want_a)):
+        y.fill_(0x7FC0)
+        ql.qlinear_stack_w4a16(ops, ws)
+        torch.cuda.synchronize()
+        check_against_oracle(host_u16(y), want, "alternating lists")
+    ql.ql_workspace_init(ws)
+    ya.fill_(0x7FC0)
+    ql.qlinear_stack_w4a16(ops_a2, ws)          # same list as the last call, but the workspace was wiped
+    ql.qlinear_stack_w4a16(ops_a, ws)
+    torch.cuda.synchronize()
+    assert ql.ql_device_status(ws) == ql.QL_OK
+    check_against_oracle(host_u16(ya), want_a, "after re-initialisation")
+    assert ql.ql_launch_count() - n0 == 7
+
+
 def test_full_verify_step_one_launch_sampled_layers(ql):
     """The benchmark's step at full size and in the launch configuration bench.py times: 36 layers
     + LM head with arg-max in ONE qlinear_stack_w4a16 call (one launch of the persistent kernel).
