@@ -346,9 +346,13 @@ __global__ void __launch_bounds__(mma_kgroups(MT) * 128 + 32, 1) qlinear_mma_ker
         for (int row = warp; row < p.M; row += 4) {
           float bv = -INFINITY;
           int bi = 0x7fffffff;
-          for (int tt = lane; tt < p.n_tiles; tt += 32) {
-            const float2 c = __ldcg(&p.ws.cand[(size_t)tt * p.m_pad + row]);
-            amax_merge(bv, bi, c.x, __float_as_int(c.y));
+          for (int t0 = lane; t0 < p.n_tiles; t0 += 32 * 8) {        // eight candidates per lane in flight
+            float2 c[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              c[q] = (t0 + 32 * q < p.n_tiles) ? __ldcg(&p.ws.cand[(size_t)(t0 + 32 * q) * p.m_pad + row]) : make_float2(-INFINITY, __int_as_float(0x7fffffff));
+#pragma unroll
+            for (int q = 0; q < 8; ++q) amax_merge(bv, bi, c[q].x, __float_as_int(c[q].y));
           }
 #pragma unroll
           for (int off = 16; off >= 1; off >>= 1) {

@@ -860,9 +860,13 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
             if (is_last && live) {
               bv = -INFINITY;
               bi = 0x7fffffff;
-              for (int tt = lane; tt < h.n_tiles; tt += 32) {
-                const float2 c = __ldcg(&sp.ws.cand[(size_t)tt * MP + rw]);
-                st_amax_merge(bv, bi, c.x, __float_as_int(c.y));
+              for (int t0 = lane; t0 < h.n_tiles; t0 += 32 * 8) {      // eight candidates per lane in flight: a round trip per 256 tiles
+                float2 c[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                  c[q] = (t0 + 32 * q < h.n_tiles) ? __ldcg(&sp.ws.cand[(size_t)(t0 + 32 * q) * MP + rw]) : make_float2(-INFINITY, __int_as_float(0x7fffffff));
+#pragma unroll
+                for (int q = 0; q < 8; ++q) st_amax_merge(bv, bi, c[q].x, __float_as_int(c[q].y));
               }
 #pragma unroll
               for (int off = 16; off >= 1; off >>= 1) {
