@@ -17,8 +17,9 @@ __host__ __device__ constexpr uint32_t align128(uint32_t x) { return (x + 127u) 
 // [0, 256)        control header: word 0 status, word 1 finished-tile counter (arg-max),
 //                 word 2 finished-CTA counter of the stack kernel, words 16-31 its per-row arg-max counters,
 //                 word 32 its counter of rows whose greedy token is final (verification tail)
-// then            per-tile arrival counters (split-K) of the single-linear kernels / partial-row flags of
-//                 the stack kernel                               [kFlagWords]
+// then            per-tile arrival counters (split-K) of the single-linear kernels [kMaxTiles], followed by the
+//                 partial-row flags of the stack kernel [2][160][16] (tagged with launch and operation, never
+//                 reset, hence in words of their own)              [kFlagWords in all]
 // then            per-operation, per-row finished-tile counters of the stack kernel, one 128-byte line each
 //                                                                [kMaxOps][16][32]
 // -- everything above is zero between calls (ql_workspace_init zeroes it once, kernels restore it) --
@@ -29,7 +30,8 @@ __host__ __device__ constexpr uint32_t align128(uint32_t x) { return (x + 127u) 
 // then            split-K partial tiles  [kMaxCtas][2 segments][2 matrices][m_pad*128] fp32
 constexpr int kMaxCtas = 320;                     // up to two CTAs per SM
 constexpr int kMaxTiles = 4096;                   // N <= 128 * 4096
-constexpr int kFlagWords = 8192;                  // tile counters / partial-row flags: [2 parities][160 CTAs][16 rows] fit
+constexpr int kStackFlagWords = 2 * 160 * 16;      // partial-row flags of the stack kernel: [2 sets][160 CTAs][16 rows]
+constexpr int kFlagWords = kMaxTiles + kStackFlagWords + 1024;   // tile counters [kMaxTiles], then the stack kernel's flags (tagged, never reset: they must not alias the counters), then spare
 constexpr int kMaxOps = 256;                      // fused operations per stack-kernel launch
 constexpr int kOpDoneStride = 32;                 // ints between the counters of two rows (one line each: they are polled)
 constexpr int kOpDescBytes = 160;

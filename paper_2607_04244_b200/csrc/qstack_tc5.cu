@@ -746,7 +746,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
         if ((sp.ablate & 8) && !whole && !finish) { pos += nch; continue; }
         pos += nch;
         const int nmat = dual ? 2 : 1;
-        int* row_flag = sp.ws.tile_cnt + (j & 1) * (16 * kSetCtas) + rw;   // flag of (CTA i, row r) at [16 i + r] of the set j & 1
+        int* row_flag = sp.ws.tile_cnt + kMaxTiles + (j & 1) * (16 * kSetCtas) + rw;   // flag of (CTA i, row r) at [16 i + r] of the set j & 1, behind the tile counters of the single-launch kernels
         float* set_slots = sp.ws.slots + (size_t)(j & 1) * kSetCtas * kSlotWords;
         float* my_slot = set_slots + (size_t)cta * kSlotWords;
 

@@ -243,6 +243,30 @@ def test_repeated_and_alternating_calls_with_one_workspace(ql):
     assert ql.ql_launch_count() - n0 == 7
 
 
+@pytest.mark.parametrize("path_name", ["MMA", "TC5"])
+def test_one_workspace_for_stack_and_single_launch_calls(ql, path_name):
+    """The stack kernel leaves its (tagged) partial-row flags behind; the tile counters of the
+    single-launch kernels must not see them, and the other way round."""
+    M, g, K, N = 16, 128, 512, 9728                       # 76 tiles: more tiles than a thread block has flag words
+    a = qsynth.make_linear([94, 0], M, K, N, g)
+    pa, xa = pack_on_device(ql, a), dev_u16(a["x"])
+    want = orc.qlinear_f64(a["x"], a["wq"], a["scale"], a["zero"], g)
+    ws = ql.new_workspace(M, N)
+    path = getattr(ql, "QL_PATH_" + path_name)
+    y = torch.full((M, N), 0x7FC0, dtype=torch.int16, device="cuda")
+    ops = ql.make_ops([dict(kind=ql.QL_OP_LINEAR, M=M, K=K, N=N, g=g, ld_in=K, ld_out=N, packed=pa, in0=xa, out=y)])
+    for order in ("stack, single", "single, stack", "stack, stack, single"):
+        for what in order.split(", "):
+            y.fill_(0x7FC0)
+            if what == "stack":
+                ql.qlinear_stack_w4a16(ops, ws)
+            else:
+                ql.qlinear_w4a16(pa, xa, y, None, M, K, N, g, ws, path=path)
+            torch.cuda.synchronize()
+            assert ql.ql_device_status(ws) == ql.QL_OK
+            check_against_oracle(host_u16(y), want, f"{what} call in the order [{order}]")
+
+
 def test_full_verify_step_one_launch_sampled_layers(ql):
     """The benchmark's step at full size and in the launch configuration bench.py times: 36 layers
     + LM head with arg-max in ONE qlinear_stack_w4a16 call (one launch of the persistent kernel).
