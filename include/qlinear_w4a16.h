@@ -199,8 +199,9 @@ int ql_linear_plan(int M, int K, int N, int g, int path, int out[4]);
  * A call that resolves to one launch of the persistent kernel is remembered per host thread: the
  * same call again (byte-identical operation list, same workspace, size and stream, and nothing
  * staged into any workspace by any thread in between) skips planning and the descriptor copy and
- * only launches.  A changed field of an operation, another list, ql_workspace_init or any
- * ql_debug_* setter makes the next call plan again.
+ * only launches.  A changed field of an operation, another list, ql_workspace_init, a
+ * qattn_swa_bf16 call or any ql_debug_* setter makes the next call plan again.  (The workspace
+ * belongs to the library between calls: a caller that writes into it must call ql_workspace_init.)
  * Errors: as qlinear_w4a16, reported for the first offending operation; nothing is launched
  * unless every operation validates.
  */

@@ -555,6 +555,7 @@ int qattn_swa_bf16(const uint16_t* Q, const uint16_t* K, const uint16_t* V, uint
   p.Q = Q; p.K = K; p.V = V; p.out = out;
   p.counters = static_cast<int*>(workspace);
   p.part = reinterpret_cast<float*>(static_cast<char*>(workspace) + kAttnCounterBytes);
+  g_desc_gen.fetch_add(1, std::memory_order_relaxed);     // the memory may once have held a stack call's descriptors
   if (launch_attn_swa(p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return QL_ERR_CUDA;
   g_launches.fetch_add(1, std::memory_order_relaxed);
   return QL_OK;
