@@ -15,8 +15,7 @@ __host__ __device__ constexpr uint32_t align128(uint32_t x) { return (x + 127u) 
 
 // ---- workspace layout -----------------------------------------------------------------------
 // [0, 256)        control header: word 0 status, word 1 finished-tile counter (arg-max),
-//                 word 2 finished-CTA counter of the stack kernel, words 16-31 its per-row arg-max counters,
-//                 word 32 its counter of rows whose greedy token is final (verification tail)
+//                 word 2 finished-CTA counter of the stack kernel
 // then            per-tile arrival counters (split-K) of the single-linear kernels [kMaxTiles], followed by the
 //                 partial-row flags of the stack kernel [2][160][16] (tagged with launch and operation, never
 //                 reset, hence in words of their own)              [kFlagWords in all]
@@ -31,7 +30,7 @@ __host__ __device__ constexpr uint32_t align128(uint32_t x) { return (x + 127u) 
 constexpr int kMaxCtas = 320;                     // up to two CTAs per SM
 constexpr int kMaxTiles = 4096;                   // N <= 128 * 4096
 constexpr int kStackFlagWords = 2 * 160 * 16;      // partial-row flags of the stack kernel: [2 sets][160 CTAs][16 rows]
-constexpr int kFlagWords = kMaxTiles + kStackFlagWords + 1024;   // tile counters [kMaxTiles], then the stack kernel's flags (tagged, never reset: they must not alias the counters), then spare
+constexpr int kFlagWords = kMaxTiles + kStackFlagWords + 1024;   // tile counters [kMaxTiles], then the stack kernel's flags (tagged, never reset: they must not alias the counters), then its 16 per-row arg-max counters and its verification-tail counter on lines of their own
 constexpr int kMaxOps = 256;                      // fused operations per stack-kernel launch
 constexpr int kOpDoneStride = 32;                 // ints between the counters of two rows (one line each: they are polled)
 constexpr int kOpDescBytes = 160;

@@ -355,7 +355,7 @@ __global__ void __launch_bounds__(kTcThreads, (MPAD == 16 ? 2 : 1)) qlinear_tc5_
             const float2 c = s_amax[q * 64 + tid];
             tc_amax_merge(bv, bi, c.x, __float_as_int(c.y));
           }
-          __stcg(&p.ws.cand[(size_t)T * p.m_pad + tid], make_float2(bv, __int_as_float(bi)));
+          __stcg(&p.ws.cand[(size_t)tid * p.n_tiles + T], make_float2(bv, __int_as_float(bi)));   // [row][tile]
         }
         __threadfence();
         named_bar_sync(2, 128);
@@ -375,7 +375,7 @@ __global__ void __launch_bounds__(kTcThreads, (MPAD == 16 ? 2 : 1)) qlinear_tc5_
               float2 c[8];
 #pragma unroll
               for (int q = 0; q < 8; ++q)
-                c[q] = (t0 + 32 * q < p.n_tiles) ? __ldcg(&p.ws.cand[(size_t)(t0 + 32 * q) * p.m_pad + row]) : make_float2(-INFINITY, __int_as_float(0x7fffffff));
+                c[q] = (t0 + 32 * q < p.n_tiles) ? __ldcg(&p.ws.cand[(size_t)row * p.n_tiles + t0 + 32 * q]) : make_float2(-INFINITY, __int_as_float(0x7fffffff));
 #pragma unroll
               for (int q = 0; q < 8; ++q) tc_amax_merge(bv, bi, c[q].x, __float_as_int(c[q].y));
             }

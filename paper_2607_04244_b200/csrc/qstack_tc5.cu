@@ -567,6 +567,9 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
     const uint32_t a_addr = tlane + w * AH * AHC;
     const uint32_t d_addr = tlane + D_COL0 + 2 * w * MP;
     constexpr uint32_t kSetCtas = kMaxCtas / 2;          // partial-tile slots and row flags: two sets of 160
+    // per-row arg-max counters (rows 0..15) and the verification-tail counter (16), one 128-byte line each:
+    // every CTA adds to them at about the same moment, and atomics on one line are served one after the other
+    int* const amax_cnt = sp.ws.tile_cnt + kMaxTiles + kStackFlagWords;
     uint32_t stg = 0, sph = 0;                          // ring stage / phase of the next sub-chunk (any group's)
     uint32_t kloc = 0;                                  // chunks this group has handed to the tensor core
     uint32_t hs = 0;                                    // half-chunks this group has stored
@@ -848,12 +851,18 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
             int is_last = 0;
             ++am_tiles;
             if (lane == 0) {
-              __stcg(&sp.ws.cand[(size_t)T * MP + rw], make_float2(bv, __int_as_float(bi)));
+              __stcg(&sp.ws.cand[(size_t)rw * h.n_tiles + T], make_float2(bv, __int_as_float(bi)));   // [row][tile]: the final reduction reads a row contiguously
               if (pos == end) {
+                // release with a fence of its own, then a RELAXED atomic: 148 acquire-release atomics on one
+                // address are served one after the other at ~0.1 us each
                 int old;
-                asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], %2;" : "=r"(old) : "l"(sp.ws.status + 16 + rw), "r"(am_tiles) : "memory");
+                fence_gpu();
+                asm volatile("atom.add.relaxed.gpu.global.s32 %0, [%1], %2;" : "=r"(old) : "l"(amax_cnt + rw * 32), "r"(am_tiles) : "memory");
                 is_last = (old + am_tiles == h.n_tiles);
-                if (is_last) sp.ws.status[16 + rw] = 0;
+                if (is_last) {
+                  fence_gpu();                           // acquire: the other CTAs' candidates
+                  amax_cnt[rw * 32] = 0;
+                }
               }
             }
             is_last = __shfl_sync(0xffffffffu, is_last, 0);
@@ -864,7 +873,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
                 float2 c[8];
 #pragma unroll
                 for (int q = 0; q < 8; ++q)
-                  c[q] = (t0 + 32 * q < h.n_tiles) ? __ldcg(&sp.ws.cand[(size_t)(t0 + 32 * q) * MP + rw]) : make_float2(-INFINITY, __int_as_float(0x7fffffff));
+                  c[q] = (t0 + 32 * q < h.n_tiles) ? __ldcg(&sp.ws.cand[(size_t)rw * h.n_tiles + t0 + 32 * q]) : make_float2(-INFINITY, __int_as_float(0x7fffffff));
 #pragma unroll
                 for (int q = 0; q < 8; ++q) st_amax_merge(bv, bi, c[q].x, __float_as_int(c[q].y));
               }
@@ -880,8 +889,11 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
               // own token at the first disagreement.
               if (dsc.draft_ids != nullptr) {
                 int rows_done = 0;
-                if (lane == 0)
-                  asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(rows_done) : "l"(sp.ws.status + 32) : "memory");
+                if (lane == 0) {
+                  fence_gpu();                           // release: this row's token
+                  asm volatile("atom.add.relaxed.gpu.global.s32 %0, [%1], 1;" : "=r"(rows_done) : "l"(amax_cnt + 16 * 32) : "memory");
+                  if (rows_done == sp.M - 1) fence_gpu();   // acquire: the other rows' tokens
+                }
                 rows_done = __shfl_sync(0xffffffffu, rows_done, 0);
                 if (rows_done == sp.M - 1) {
                   const int tok = lane < sp.M ? (lane == rw ? bi : __ldcg(&argmax_out[lane])) : -1;
@@ -892,7 +904,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
                   if (lane == 0) {
                     dsc.accept_out[0] = a;
                     dsc.accept_out[1] = a < sp.M ? bonus : -1;
-                    sp.ws.status[32] = 0;
+                    amax_cnt[16 * 32] = 0;
                   }
                 }
               }
@@ -940,8 +952,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
     old = __shfl_sync(0xffffffffu, old, 0);
     if (old == (int)gridDim.x - 1) {
       for (int i = lane; i < sp.n_ops * 16; i += 32) sp.ws.op_done[(size_t)i * kOpDoneStride] = 0;
-      if (lane < 16) sp.ws.status[16 + lane] = 0;              // per-row arg-max counters
-      if (lane == 16) sp.ws.status[32] = 0;                    // verification-tail row counter
+      if (lane <= 16) sp.ws.tile_cnt[kMaxTiles + kStackFlagWords + lane * 32] = 0;   // per-row arg-max counters, verification-tail row counter
       if (lane == 0) { *sp.ws.amax_done = 0; *sp.ws.exit_cnt = 0; }
     }
   }
