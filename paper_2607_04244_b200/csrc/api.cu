@@ -197,8 +197,6 @@ static bool independent_ops(const MegaOp& prev, const MegaOp& cur, int M) {
   return true;
 }
 
-constexpr int kBatchMaxGroups = 24;   // K <= 24 groups: X of one operation (24 x 4.25 KB) beside a useful ring
-
 // True if the run is a list of plain linears no two of which share a buffer other than inputs
 // that both only read: nothing in it has to wait for a result.
 static bool independent_run(const std::vector<MegaOp>& mega, int M) {
@@ -210,12 +208,15 @@ static bool independent_run(const std::vector<MegaOp>& mega, int M) {
       if (!independent_ops(mega[a], mega[b], M) || !independent_ops(mega[b], mega[a], M)) return false;
   return true;
 }
+
 // An independent run is laid end to end and cut into one piece per CTA if the X of a whole
-// operation fits in shared memory (a piece spans whole tile columns).
-static bool fits_one_stream(const std::vector<MegaOp>& mega) {
-  for (const MegaOp& m : mega)
-    if (m.n_groups > kBatchMaxGroups) return false;
-  return true;
+// operation (a piece spans whole tile columns) fits in shared memory beside a ring of at least
+// six stages: the shared-memory plan of the run, with its split fields set for one stream, says so.
+static bool plan_one_stream(std::vector<MegaOp>& mega, int ncta, int g, int sms) {
+  uint32_t total = 0;
+  for (MegaOp& m : mega) { m.cat_base = total; total += m.total_chunks; }
+  for (MegaOp& m : mega) run_split(total, (uint32_t)ncta, m.nc, m.cq, m.cr);
+  return stack_plan(mega.data(), (int)mega.size(), g, sms).ok;
 }
 
 static bool is_dual(const ql_op* ops, int i, int n_ops) {
@@ -274,11 +275,9 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
       // takes one contiguous piece.  Anything else is a chain: every operation is its own run and
       // waits for the one before it.
       const bool indep = independent_run(mega, run_M);
-      const bool batch = indep && fits_one_stream(mega);
+      const bool batch = indep && plan_one_stream(mega, ncta, run_g, sms);
       if (batch) {
-        uint32_t total = 0;
-        for (MegaOp& m : mega) { m.cat_base = total; total += m.total_chunks; }
-        for (MegaOp& m : mega) { run_split(total, (uint32_t)ncta, m.nc, m.cq, m.cr); m.flags |= kOpLazy; }
+        for (MegaOp& m : mega) m.flags |= kOpLazy;
       } else {
         for (size_t j = 0; j < mega.size(); ++j) {
           MegaOp& m = mega[j];

@@ -1,6 +1,7 @@
 """GPU parity of qlinear_stack_w4a16 on lists of INDEPENDENT linears (no two share a buffer other
 than inputs both only read).  Such a list is not a chain: the launcher lays the operations' chunks
-end to end and cuts them into one contiguous piece per thread block (K of at most 24 groups), or
+end to end and cuts them into one contiguous piece per thread block (where the X operand of a whole
+tile fits in shared memory beside the weight ring), or
 splits every operation among all thread blocks without waiting for its predecessor (longer K).
 Every output is compared with the oracle element by element at the library's tolerances."""
 import numpy as np
@@ -36,9 +37,9 @@ def run_independent(ql, lins, M, g, n_max, shared_x=None, runs=1):
     return plan, outs
 
 
-@pytest.mark.parametrize("name", ["gate", "qkv"])
+@pytest.mark.parametrize("name", ["gate", "qkv", "o"])
 def test_bench_shapes_one_stream(ql, name):
-    """The benchmark's gate/up and fused-qkv shapes at M=16, g=128, four distinct weight sets each:
+    """The benchmark's gate/up, fused-qkv and o shapes at M=16, g=128, four distinct weight sets each:
     one launch, the operations run as one stream of chunks (thread blocks' pieces cross operation
     boundaries and split tiles in the middle)."""
     M, g = 16, 128
@@ -53,18 +54,20 @@ def test_bench_shapes_one_stream(ql, name):
         assert np.array_equal(outs[0][i], outs[1][i]), "second run differs"
 
 
-@pytest.mark.parametrize("name", ["down", "o"])
-def test_bench_shapes_long_k(ql, name):
-    """down (K = 76 groups) and o (32 groups): too long for one stream, so every operation is split
-    among all thread blocks, none waits for its predecessor."""
+@pytest.mark.parametrize("n_lin,one_stream", [(3, True), (5, False)])
+def test_down_shape_short_and_long_lists(ql, n_lin, one_stream):
+    """down (K = 76 groups).  Three of them give every thread block a piece of 31 chunks: the X
+    operand of those groups fits in shared memory and the list runs as one stream.  Five give
+    pieces of 52 chunks, whose X does not fit beside the weight ring: every operation is then
+    split among all thread blocks, none waits for its predecessor."""
     M, g = 16, 128
-    K, N = qsynth.LAYER_SHAPES[name]
-    lins = [qsynth.make_linear([78, i, K, N], M, K, N, g) for i in range(3)]
+    K, N = qsynth.LAYER_SHAPES["down"]
+    lins = [qsynth.make_linear([78, i, K, N], M, K, N, g) for i in range(n_lin)]
     plan, outs = run_independent(ql, lins, M, g, N, runs=2)
-    assert plan["stack_launches"] == 1 and plan["batch_launches"] == 0 and plan["independent"] == 2
+    assert plan["stack_launches"] == 1 and plan["batch_launches"] == (1 if one_stream else 0) and plan["independent"] == n_lin - 1
     for i, d in enumerate(lins):
         y64 = orc.qlinear_f64(d["x"], d["wq"], d["scale"], d["zero"], g, col_block=4096)
-        check_against_oracle(outs[0][i], y64, f"{name} #{i}")
+        check_against_oracle(outs[0][i], y64, f"down #{i} of {n_lin}")
         assert np.array_equal(outs[0][i], outs[1][i]), "second run differs"
 
 
