@@ -188,9 +188,9 @@ int ql_linear_plan(int M, int K, int N, int g, int path, int out[4]);
  * it runs: a linear may start streaming its weights while the operation before it finishes.
  * Runs of operations with M <= 16 and one group size execute as ONE cooperative launch of a
  * persistent kernel.  A run of plain linears no two of which share a buffer (other than inputs
- * both only read) and whose X operand for a whole tile fits in shared memory beside the weight
- * ring (K up to about 32 groups) is treated as one long stream of chunks cut into one contiguous
- * piece per thread block; any other run is a chain - glue folded into the
+ * both only read) is treated as one long stream of chunks cut into one contiguous piece per
+ * thread block (the X operand stays in shared memory per operation where it fits and follows the
+ * chunks through a ring of slots where it does not); any other run is a chain - glue folded into the
  * neighbouring linears, gate/up pairs fused, every operation waiting for the one before it.  The
  * thread blocks wait for one another with bounded waits, so a stream that is starved of SMs for
  * more than 2 s reports QL_ERR_DEVICE_TIMEOUT in the status word instead of hanging.

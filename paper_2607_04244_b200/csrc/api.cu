@@ -16,9 +16,9 @@ cudaError_t launch_attn_swa(const AttnParams&, cudaStream_t);
 size_t plan_linear_mma(LinearParams&);
 cudaError_t launch_linear_tc5(LinearParams, int sms, cudaStream_t, bool pdl);
 bool tc5_supported(const LinearParams&, int sms);
-struct StackPlan { int ncta, n_x, n_stages; size_t smem; bool ok; };
+struct StackPlan { int ncta, n_x, n_stages, x_ring; size_t smem; bool ok; };
 int stack_ncta(int sms);
-StackPlan stack_plan(const MegaOp* ops, int n_ops, int g, int sms);
+StackPlan stack_plan(const MegaOp* ops, int n_ops, int g, int sms, bool one_stream = false);
 cudaError_t launch_stack_tc5(const StackParams& sp, int g, size_t smem, cudaStream_t stream);
 cudaError_t launch_unit_rms(const uint16_t*, const uint16_t*, uint16_t*, int, int, int, int, bool, cudaStream_t);
 
@@ -209,14 +209,11 @@ static bool independent_run(const std::vector<MegaOp>& mega, int M) {
   return true;
 }
 
-// An independent run is laid end to end and cut into one piece per CTA if the X of a whole
-// operation (a piece spans whole tile columns) fits in shared memory beside a ring of at least
-// six stages: the shared-memory plan of the run, with its split fields set for one stream, says so.
-static bool plan_one_stream(std::vector<MegaOp>& mega, int ncta, int g, int sms) {
+// An independent run is laid end to end and cut into one contiguous piece per CTA.
+static void split_one_stream(std::vector<MegaOp>& mega, int ncta) {
   uint32_t total = 0;
   for (MegaOp& m : mega) { m.cat_base = total; total += m.total_chunks; }
   for (MegaOp& m : mega) run_split(total, (uint32_t)ncta, m.nc, m.cq, m.cr);
-  return stack_plan(mega.data(), (int)mega.size(), g, sms).ok;
 }
 
 static bool is_dual(const ql_op* ops, int i, int n_ops) {
@@ -275,30 +272,31 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
       // takes one contiguous piece.  Anything else is a chain: every operation is its own run and
       // waits for the one before it.
       const bool indep = independent_run(mega, run_M);
-      const bool batch = indep && plan_one_stream(mega, ncta, run_g, sms);
+      const bool batch = indep;
+      bool x_ring = false;
       if (batch) {
+        split_one_stream(mega, ncta);
         for (MegaOp& m : mega) m.flags |= kOpLazy;
+        // X resident per operation where it fits (faster: no per-chunk hand-over), else through the ring
+        x_ring = !stack_plan(mega.data(), (int)mega.size(), run_g, sms, false).ok;
       } else {
         for (size_t j = 0; j < mega.size(); ++j) {
           MegaOp& m = mega[j];
           m.cat_base = 0;
           run_split(m.total_chunks, (uint32_t)ncta, m.nc, m.cq, m.cr);
-          // independent operations whose K is too long for one stream: each is split among all CTAs
-          // like a chained one, but waits only for the operation two back
-          if (indep) { if (j > 1) m.flags |= kOpWait2; }
-          else if (j > 0) m.flags |= kOpWait;
+          if (j > 0) m.flags |= kOpWait;
         }
       }
       const int hook = g_no_release_op.load(std::memory_order_relaxed);
       if (hook >= 0 && hook < (int)mega.size()) mega[hook].flags |= kOpNoRelease;
-      StackPlan plan = stack_plan(mega.data(), (int)mega.size(), run_g, sms);
+      StackPlan plan = stack_plan(mega.data(), (int)mega.size(), run_g, sms, x_ring);
       if (!plan.ok) return QL_ERR_UNSUPPORTED;   // cannot happen: every operation was checked when it was added
       int n_tiles_cap = 1;
       for (const MegaOp& m : mega) n_tiles_cap = m.n_tiles > n_tiles_cap ? m.n_tiles : n_tiles_cap;
       StackParams sp = {};
       sp.ws = ws_carve(workspace, n_tiles_cap, 16);
       sp.ops = reinterpret_cast<const MegaOp*>(sp.ws.desc);
-      sp.n_ops = (int)mega.size(); sp.M = run_M; sp.ncta = plan.ncta; sp.n_stages = plan.n_stages; sp.n_x = plan.n_x;
+      sp.n_ops = (int)mega.size(); sp.M = run_M; sp.ncta = plan.ncta; sp.n_stages = plan.n_stages; sp.n_x = plan.n_x; sp.x_ring = plan.x_ring;
       sp.wait_ns = g_wait_ns.load(std::memory_order_relaxed);
       sp.ablate = g_ablate.load(std::memory_order_relaxed);
       sp.timeline = g_timeline.load(std::memory_order_relaxed);

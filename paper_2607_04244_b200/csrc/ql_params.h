@@ -36,7 +36,6 @@ struct LinearParams {
 // The first 32 bytes hold what every role reads at every operation.
 constexpr int kOpDual = 1;        // two matrices (packed0, packed1) share X
 constexpr int kOpWait = 2;        // X may be read only after operation j-1 has finished every tile
-constexpr int kOpWait2 = 8;       // X may be read only after operation j-2 has finished (its partial-tile slots are reused)
 constexpr int kOpLazy = 16;       // nothing in the launch waits for this operation's tiles: they need not be published, and the
                                   // next tile segment may be started before the current one is finished
 constexpr int kOpNoRelease = 4;   // test hook: finished tiles are not published (the next operation's wait runs out)
@@ -72,6 +71,8 @@ struct StackParams {
   int ncta;
   int n_stages;            // ring depth
   int n_x;                 // X slots (groups) in shared memory
+  int x_ring;              // 0: X of an operation is built once, by the unpack threads; P > 0 (one stream of independent
+                           // linears): the X slots are a ring of P chunks filled by a loader warp, chunk by chunk
   int ablate;              // timing experiments only (see the stack kernel); 0 in production
   uint32_t epoch;          // launch number: partial tiles in the workspace carry (epoch, operation) tags
   uint64_t wait_ns;        // budget of every bounded wait

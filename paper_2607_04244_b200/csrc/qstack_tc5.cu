@@ -15,6 +15,9 @@
 //          ~150 cycles while tensor-memory stores are running, and a chunk needs 8).
 //   21     watcher: polls the counter of the previous operation, so that the other warps can work
 //          while they wait, and computes the row scales 1/rms from the per-tile sums of squares.
+//   22     X loader, only for one stream of independent linears: copies the X columns of every chunk
+//          into a ring of X slots ahead of the MMAs (cp.async, completion on an mbarrier per slot),
+//          so that an operation boundary costs the unpack groups nothing and K may be of any length.
 //
 // What keeps a chain of dependent operations short (each one needs every output of the one before):
 //   * a group owns three half-chunk A buffers in tensor memory and unpacks the first one and a
@@ -46,7 +49,10 @@ constexpr int MP = 16;                                  // padded rows
 constexpr int kUnpackThreads = NWG * 128;               // 512
 constexpr int kIssuers = NWG;                           // one per group
 constexpr int kWarpProducer = NWG * 4, kWarpIssuer0 = NWG * 4 + 1, kWarpWatcher = NWG * 4 + 1 + kIssuers;
+constexpr int kWarpXLoader = kWarpWatcher + 1;           // exists only in the kernel variant with the X ring
 constexpr int kStThreads = (kWarpWatcher + 1) * 32;     // 704
+constexpr int kStThreadsRing = (kWarpXLoader + 1) * 32; // 736
+constexpr int kXRingSlots = 16;                         // X slots of the ring (one stream of independent linears)
 constexpr int kStMaxStages = 24;
 constexpr uint32_t kStSmemBudget = 232448u;
 constexpr uint32_t kXLbo = 16u * MP + 16u;              // bytes between K-adjacent 8x16-byte core matrices (+16: bank spread)
@@ -318,8 +324,10 @@ __device__ __forceinline__ void build_x(const StackParams& sp, const MegaOp& d, 
   if (lane == 0) mbar_arrive(x_full);
 }
 
-template <int G>
-__global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_constant__ StackParams sp) {
+// RING: variant for one stream of independent linears whose X does not fit per operation (one more
+// warp, the X loader; the issuers take X slot by slot).  The other variant has none of that code.
+template <int G, bool RING>
+__global__ void __launch_bounds__(RING ? kStThreadsRing : kStThreads, 1) qstack_tc5_kernel(const __grid_constant__ StackParams sp) {
   extern __shared__ __align__(1024) uint8_t smem[];
   constexpr uint32_t STAGE = align128(chunk_bytes(G));
   constexpr uint32_t XSLOT = st_xslot_bytes(G);
@@ -340,7 +348,9 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
   uint64_t* a_empty = a_full + NWG * AH;                // [NWG][AH]
   uint64_t* d_full = a_empty + NWG * AH;                // [NWG][2]
   uint64_t* x_full = d_full + NWG * 2;                  // [1]
-  float* s_inv = reinterpret_cast<float*>(x_full + 2);  // [16] 1/rms per row of the operation being prepared
+  uint64_t* xr_full = x_full + 2;                       // [kXRingSlots] X ring: the slot's columns have landed
+  uint64_t* xr_empty = xr_full + kXRingSlots;           // [kXRingSlots] the MMAs that read the slot are complete
+  float* s_inv = reinterpret_cast<float*>(xr_empty + kXRingSlots);  // [16] 1/rms per row of the operation being prepared
   int* s_flag = reinterpret_cast<int*>(s_inv + 16);     // [0..7]
   volatile int* s_abort = s_flag + 8;
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_flag + 9);
@@ -367,6 +377,10 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
     }
     for (int i = 0; i < NWG * 2; ++i) mbar_init(&d_full[i], 1);
     mbar_init(x_full, NWG * 4);
+    for (int i = 0; i < kXRingSlots; ++i) {
+      mbar_init(&xr_full[i], 32);                        // the loader's 32 lanes, each when its copies have landed
+      mbar_init(&xr_empty[i], 1);
+    }
     *s_abort = 0;
     *s_dep = 0;
     *s_invrdy = 0;
@@ -378,7 +392,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
     tmem_alloc(s_tmem, TMEM_COLS);
     tmem_relinquish();
   }
-  for (int i = tid; i < 2 * sp.n_ops; i += kStThreads)
+  for (int i = tid; i < 2 * sp.n_ops; i += (RING ? kStThreadsRing : kStThreads))
     s_heads[i] = __ldg(reinterpret_cast<const uint4*>(ops + (i >> 1)) + (i & 1));
   tc_fence_before_sync();
   __syncthreads();
@@ -456,7 +470,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
       ++pcount;
       // an operation waits for the one before it (it consumes its output), or only for the one two
       // back (independent operations: the partial-tile slots and flags alternate between two sets)
-      const int dep = (h.flags & kOpWait) ? j - 1 : ((h.flags & kOpWait2) ? j - 2 : -1);
+      const int dep = (h.flags & kOpWait) ? j - 1 : -1;
       if (dep >= 0) {
         // every tile is published row by row; lane r polls the counter of row r (one line per counter)
         if (lane < 16) {
@@ -500,6 +514,43 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
       if (*s_abort) break;
     }
     if (lane == 0 && *s_abort) { *s_descrdy = 0x7ffffff0; *s_dep = 0x7ffffff0; *s_invrdy = 0x7ffffff0; }
+  } else if (RING && warp == kWarpXLoader) {
+    // ------------------------------------------------------------------ X loader (one stream of independent linears)
+    if (sp.x_ring > 0 && !(sp.ablate & 1)) {
+      constexpr uint32_t UPR = G / 8;                     // 16-byte units per row of one group
+      const uint32_t P = (uint32_t)sp.x_ring;
+      uint32_t r = 0;                                    // ring position = chunks of this CTA so far
+      for (int j = 0; j < sp.n_ops; ++j) {
+        const OpHead h = load_head(s_heads, j);
+        uint32_t start, end;
+        op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
+        if (start >= end) continue;
+        const uint16_t* in0 = ldg_ptr(&ops[j].in0);
+        const int ld_in = __ldg(&ops[j].ld_in);
+        const uint32_t Gn = (uint32_t)h.n_groups;
+        for (uint32_t c = start; c < end; ++c, ++r) {
+          const uint32_t slot = r % P;
+          if (r >= P) {
+            if (lane == 0) st_mbar_wait(&xr_empty[slot], ((r / P) - 1) & 1, wc, 18);
+            __syncwarp();
+          }
+          if (*s_abort) break;
+          const uint32_t Gi = c % Gn;                    // the chunk's group
+          uint8_t* dst = xbuf + (size_t)slot * XSLOT;
+          // unit (row m, k-unit ku): lanes run along K, two rows per pass
+#pragma unroll
+          for (uint32_t u = (uint32_t)lane; u < (uint32_t)MP * UPR; u += 32) {
+            const uint32_t m = u / UPR, ku = u % UPR;
+            const bool live = (int)m < sp.M;
+            cp_async16(dst + ku * kXLbo + (m >> 3) * 128u + (m & 7u) * 16u,
+                       live ? (in0 + (size_t)m * ld_in + (size_t)Gi * G + ku * 8) : in0, live ? 16u : 0u);
+          }
+          cp_async_arrive_noinc(&xr_full[slot]);
+        }
+        if (*s_abort) break;
+      }
+      asm volatile("cp.async.wait_all;" ::: "memory");   // nothing of this warp is in flight when the CTA exits
+    }
   } else if (warp >= kWarpIssuer0) {
     // ------------------------------------------------------------------ MMA issue for unpack group w
     if (lane == 0) {
@@ -511,7 +562,9 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
       const uint32_t a_base = tmem + w * AH * AHC;
       uint32_t k = 0;                                  // chunks this group has handed over so far
       uint32_t hs = 0;                                 // half-chunks
-      uint32_t xops = 0;                               // operations this CTA took part in so far
+      uint32_t xops = 0;                               // operations this CTA took part in so far whose X the unpack threads built
+      uint32_t rbase = 0;                              // X ring: chunks of this CTA before the current operation
+      const uint32_t P = RING ? (uint32_t)sp.x_ring : 1u;
       QL_CYC_DECL;
       for (int j = 0; j < sp.n_ops; ++j) {
         const OpHead h = load_head(s_heads, j);
@@ -521,12 +574,20 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
         const bool dual = (h.flags & kOpDual) != 0;
         const uint32_t Gn = (uint32_t)h.n_groups;
         const uint32_t n_sub = (end - start) * (dual ? 2u : 1u);
-        ++xops;
-        if (sp.ablate & 1) continue;
-        bool first = true;
+        constexpr bool ring = RING;                    // X comes chunk by chunk from the loader warp (never with dual operations)
+        if (!ring) ++xops;
+        if (sp.ablate & 1) { rbase += end - start; continue; }
+        bool first = !ring;
         for (uint32_t e = w; e < n_sub; e += NWG, ++k) {
           uint32_t xk = dual ? (e >> 1) : e;           // X slot = chunk number within the CTA, modulo the group count
-          xk = xk % Gn;
+          if (ring) {
+            const uint32_t r = rbase + e;
+            xk = r % P;
+            st_mbar_wait(&xr_full[xk], (r / P) & 1, wc, 17);
+            fence_proxy_async();                         // the copies were generic-proxy writes; the MMAs read through the async proxy
+          } else {
+            xk = xk % Gn;
+          }
           const uint32_t d_tmem = tmem + D_COL0 + (2 * w + (k & 1)) * MP;
           const uint64_t xdesc = desc0 + (uint64_t)(xk * SLOT);
 #pragma unroll
@@ -554,7 +615,9 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
             QL_CYC_ADD(3, 1);
           }
           tc_commit(&d_full[2 * w + (k & 1)]);
+          if (ring) tc_commit(&xr_empty[xk]);            // the slot may be refilled once this chunk's MMAs are complete
         }
+        rbase += end - start;
       }
       QL_CYC_FLUSH_I();
     }
@@ -667,7 +730,7 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
       }
       QL_STAMP(1);
       // -------- X duty (all 512 threads): wait for the previous operation, build the X operand --------
-      build_x<G>(sp, dsc, j, xbuf, s_inv, s_dep, s_invrdy, x_full, wc, start, my_chunks, Gn);
+      if (!RING) build_x<G>(sp, dsc, j, xbuf, s_inv, s_dep, s_invrdy, x_full, wc, start, my_chunks, Gn);
       QL_STAMP(3);
 
       // -------- chunks of this operation --------
@@ -963,18 +1026,20 @@ __global__ void __launch_bounds__(kStThreads, 1) qstack_tc5_kernel(const __grid_
 // Shared-memory plan for a list of operations with common M <= 16 and g whose split fields are
 // set; ok = false if some operation's X does not fit beside a ring of at least 6 stages.
 struct StackPlan {
-  int ncta, n_x, n_stages;
+  int ncta, n_x, n_stages, x_ring;
   size_t smem;
   bool ok;
 };
 
 int stack_ncta(int sms) { return sms < kMaxCtas / 2 ? sms : kMaxCtas / 2; }   // one 32 KB partial slot per CTA
 
-StackPlan stack_plan(const MegaOp* ops, int n_ops, int g, int sms) {
+// x_ring: the operations are independent plain linears laid end to end whose X does not fit per operation;
+// it comes through a ring of kXRingSlots slots filled by the loader warp, whatever K is.
+StackPlan stack_plan(const MegaOp* ops, int n_ops, int g, int sms, bool one_stream) {
   StackPlan r = {};
   const int ncta = stack_ncta(sms);
   uint32_t n_x = 1;
-  for (int j = 0; j < n_ops; ++j) {
+  for (int j = 0; j < n_ops && !one_stream; ++j) {
     // the longest piece of this operation that one CTA owns
     uint32_t longest = 0;
     const uint32_t nc = ops[j].nc;
@@ -986,28 +1051,31 @@ StackPlan stack_plan(const MegaOp* ops, int n_ops, int g, int sms) {
     const uint32_t need = longest < (uint32_t)ops[j].n_groups ? longest : (uint32_t)ops[j].n_groups;
     if (need > n_x) n_x = need;
   }
+  if (one_stream) n_x = kXRingSlots;
   const uint32_t stage = align128(chunk_bytes(g)), xslot = st_xslot_bytes(g);
   const uint32_t fixed = st_fixed_smem() + 32u * (uint32_t)n_ops;   // + the head table
   if (fixed + n_x * xslot + 6 * stage > kStSmemBudget) return r;
   int ns = (int)((kStSmemBudget - fixed - n_x * xslot) / stage);
   if (ns > kStMaxStages) ns = kStMaxStages;
-  r.ncta = ncta; r.n_x = (int)n_x; r.n_stages = ns;
+  r.ncta = ncta; r.n_x = (int)n_x; r.n_stages = ns; r.x_ring = one_stream ? kXRingSlots : 0;
   r.smem = (size_t)ns * stage + (size_t)n_x * xslot + fixed;
   r.ok = true;
   return r;
 }
 
-template <int G>
+template <int G, bool RING>
 static cudaError_t stack_launch_g(const StackParams& sp, size_t smem, cudaStream_t stream) {
   // all CTAs wait on one another's progress: they must be co-resident (the cooperative launch checks it)
-  cudaError_t e = cudaFuncSetAttribute(qstack_tc5_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStSmemBudget);
+  cudaError_t e = cudaFuncSetAttribute(qstack_tc5_kernel<G, RING>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStSmemBudget);
   if (e != cudaSuccess) return e;
   void* args[] = {const_cast<StackParams*>(&sp)};
-  return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(qstack_tc5_kernel<G>), dim3(sp.ncta), dim3(kStThreads), args, smem, stream);
+  return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(qstack_tc5_kernel<G, RING>), dim3(sp.ncta),
+                                     dim3(RING ? kStThreadsRing : kStThreads), args, smem, stream);
 }
 
 cudaError_t launch_stack_tc5(const StackParams& sp, int g, size_t smem, cudaStream_t stream) {
-  return g == 128 ? stack_launch_g<128>(sp, smem, stream) : stack_launch_g<64>(sp, smem, stream);
+  if (sp.x_ring > 0) return g == 128 ? stack_launch_g<128, true>(sp, smem, stream) : stack_launch_g<64, true>(sp, smem, stream);
+  return g == 128 ? stack_launch_g<128, false>(sp, smem, stream) : stack_launch_g<64, false>(sp, smem, stream);
 }
 
 }  // namespace ql

@@ -1,8 +1,7 @@
 """GPU parity of qlinear_stack_w4a16 on lists of INDEPENDENT linears (no two share a buffer other
 than inputs both only read).  Such a list is not a chain: the launcher lays the operations' chunks
-end to end and cuts them into one contiguous piece per thread block (where the X operand of a whole
-tile fits in shared memory beside the weight ring), or
-splits every operation among all thread blocks without waiting for its predecessor (longer K).
+end to end and cuts them into one contiguous piece per thread block; the X operand follows the
+chunks through a ring of slots.
 Every output is compared with the oracle element by element at the library's tolerances."""
 import numpy as np
 import pytest
@@ -54,17 +53,16 @@ def test_bench_shapes_one_stream(ql, name):
         assert np.array_equal(outs[0][i], outs[1][i]), "second run differs"
 
 
-@pytest.mark.parametrize("n_lin,one_stream", [(3, True), (5, False)])
-def test_down_shape_short_and_long_lists(ql, n_lin, one_stream):
-    """down (K = 76 groups).  Three of them give every thread block a piece of 31 chunks: the X
-    operand of those groups fits in shared memory and the list runs as one stream.  Five give
-    pieces of 52 chunks, whose X does not fit beside the weight ring: every operation is then
-    split among all thread blocks, none waits for its predecessor."""
+@pytest.mark.parametrize("n_lin", [3, 7])
+def test_down_shape_long_k(ql, n_lin):
+    """down (K = 76 groups): the X operand of a whole tile (330 KB) cannot be resident, it comes through
+    the ring of X slots chunk by chunk.  Three linears give every thread block a piece of 31 chunks,
+    seven a piece of 72: both shorter than a tile, the pieces cross tile and operation boundaries."""
     M, g = 16, 128
     K, N = qsynth.LAYER_SHAPES["down"]
     lins = [qsynth.make_linear([78, i, K, N], M, K, N, g) for i in range(n_lin)]
     plan, outs = run_independent(ql, lins, M, g, N, runs=2)
-    assert plan["stack_launches"] == 1 and plan["batch_launches"] == (1 if one_stream else 0) and plan["independent"] == n_lin - 1
+    assert plan["stack_launches"] == 1 and plan["batch_launches"] == 1 and plan["independent"] == n_lin - 1
     for i, d in enumerate(lins):
         y64 = orc.qlinear_f64(d["x"], d["wq"], d["scale"], d["zero"], g, col_block=4096)
         check_against_oracle(outs[0][i], y64, f"down #{i} of {n_lin}")

@@ -75,17 +75,11 @@ def test_independent_linears_skip_the_wait_but_write_after_write_does_not(ql):
     # independent of the neighbour but not pairwise (ops 0 and 2 write the same buffer): a chain
     c = plan(ql, [lin(0, buf(20)), lin(1, buf(21)), lin(2, buf(20))])
     assert c["independent"] == 0 and c["batch_launches"] == 0
-    # K = 76 groups: the X of a whole tile would not fit in shared memory, so every
-    # operation is split among all thread blocks; independent ones wait only for the one two back
+    # any K runs as one stream: the X operand comes chunk by chunk through a ring of slots
     def wide(i):
         return dict(kind=0, M=16, K=9728, N=2560, g=128, ld_in=9728, ld_out=2560, packed=buf(100 + i), in0=buf(1), out=buf(20 + i))
-    c = plan(ql, [wide(i) for i in range(4)])
-    assert c["fused_ops"] == 4 and c["batch_launches"] == 0 and c["independent"] == 3
-    # K = 32 groups still fits beside a six-stage ring: one stream
-    def o_like(i):
-        return dict(kind=0, M=16, K=4096, N=2560, g=128, ld_in=4096, ld_out=2560, packed=buf(100 + i), in0=buf(1), out=buf(20 + i))
-    c = plan(ql, [o_like(i) for i in range(4)])
-    assert c["batch_launches"] == 1
+    c = plan(ql, [wide(i) for i in range(40)])
+    assert c["fused_ops"] == 40 and c["batch_launches"] == 1 and c["independent"] == 39
     # a linear that reads its predecessor's output is dependent
     a = dict(kind=0, M=16, K=2560, N=2560, g=128, ld_in=2560, ld_out=2560, packed=buf(100), in0=buf(1), out=buf(2))
     b = dict(kind=0, M=16, K=2560, N=2560, g=128, ld_in=2560, ld_out=2560, packed=buf(101), in0=buf(2), out=buf(3))
