@@ -186,25 +186,20 @@ class VerifyStep:
 
 def independent_point(ql, torch, M, K, N, g, packed, ws, sym=False, iters=5):
     """Throughput of one linear shape with cold L2: the distinct weight sets `packed` (together more
-    than twice the L2), one input, DISTINCT outputs, back to back.  Up to 16 rows the whole list
-    is one qlinear_stack_w4a16 call (independent operations: nothing waits for a result); above,
-    qlinear_w4a16 is launched once per weight set.  Returns microseconds per linear and the kernel."""
+    than twice the L2), one input, DISTINCT outputs, back to back: the whole list is one
+    qlinear_stack_w4a16 call (independent operations: nothing waits for a result; above 16 rows the
+    launcher cuts every linear into slabs of 16 rows).  Returns microseconds per linear and the kernel."""
     R = len(packed)
     xin = torch.randn((M, K), device="cuda").to(torch.bfloat16).view(torch.int16)
     youts = [torch.zeros((M, N), dtype=torch.int16, device="cuda") for _ in range(R)]
-    if M <= 16:
-        ops = ql.make_ops([dict(kind=ql.QL_OP_LINEAR, M=M, K=K, N=N, g=g, ld_in=K, ld_out=N, packed=p, in0=xin, out=y)
-                           for p, y in zip(packed, youts)])
-        plan = ql.ql_stack_plan(ops, ws.data_ptr(), ws.numel())
-        fn = lambda: ql.qlinear_stack_w4a16(ops, ws)
-        kernel = "qstack_tc5_kernel, one stream of chunks" if plan["batch_launches"] else \
-            "qstack_tc5_kernel, every operation split over all SMs, no wait on the predecessor"
+    ops = ql.make_ops([dict(kind=ql.QL_OP_LINEAR, M=M, K=K, N=N, g=g, ld_in=K, ld_out=N, packed=p, in0=xin, out=y)
+                       for p, y in zip(packed, youts)])
+    plan = ql.ql_stack_plan(ops, ws.data_ptr(), ws.numel())
+    fn = lambda: ql.qlinear_stack_w4a16(ops, ws)
+    if plan["batch_launches"] == plan["stack_launches"] == 1 and plan["single_linears"] == 0:
+        kernel = "qstack_tc5_kernel, one stream of chunks" + ("" if M <= 16 else f", {(M + 15) // 16} slabs of 16 rows per linear")
     else:
-        def fn():
-            for p, y in zip(packed, youts):
-                ql.qlinear_w4a16(p, xin, y, None, M, K, N, g, ws)
-        name = ql.PATH_NAMES[ql.ql_select_path(M, K, N, g)]
-        kernel = ("qlinear_tc5_kernel" if name == "tcgen05" else "qlinear_mma_kernel") + ", one launch per linear"
+        kernel = f"planner: {plan}"
     for _ in range(3):
         fn()
     torch.cuda.synchronize()

@@ -187,7 +187,10 @@ int ql_linear_plan(int M, int K, int N, int g, int path, int out[4]);
  * The packed weights of every LINEAR must be complete before the call and must not change while
  * it runs: a linear may start streaming its weights while the operation before it finishes.
  * Runs of operations with M <= 16 and one group size execute as ONE cooperative launch of a
- * persistent kernel.  A run of plain linears no two of which share a buffer (other than inputs
+ * persistent kernel.  A list that consists of pairwise independent plain linears with one common
+ * M above 16 does too: every linear is cut into slabs of 16 rows, which join the one stream of
+ * chunks (the weights are unpacked once per slab).  Other operations with M > 16 are launched
+ * one by one.  A run of plain linears no two of which share a buffer (other than inputs
  * both only read) is treated as one long stream of chunks cut into one contiguous piece per
  * thread block (the X operand stays in shared memory per operation where it fits and follows the
  * chunks through a ring of slots where it does not); any other run is a chain - glue folded into the

@@ -162,6 +162,7 @@ static MegaOp make_mega(const ql_op& o, const ql_op* second) {
   m.xout = nullptr; m.argmax_out = o.argmax_out;
   m.draft_ids = o.draft_ids; m.accept_out = o.accept_out;
   m.K = o.K; m.N = o.N; m.ld_in = o.ld_in; m.ld_out = o.ld_out; m.ld_xout = 0;
+  m.rows = o.M;
   m.n_tiles = o.N / kTileN; m.n_groups = o.K / o.g;
   m.total_chunks = (uint32_t)m.n_tiles * (uint32_t)m.n_groups;
   m.flags = second ? kOpDual : 0;
@@ -181,13 +182,13 @@ static Span span_of(const void* p, int M, int ld, int n, int elt) {
 static bool overlap(Span a, Span b) { return a.lo < b.hi && b.lo < a.hi; }
 
 // True if `cur` neither reads nor overwrites anything `prev` writes, nor overwrites what it reads.
-static bool independent_ops(const MegaOp& prev, const MegaOp& cur, int M) {
+static bool independent_ops(const MegaOp& prev, const MegaOp& cur) {
   if (cur.prologue != 0 || prev.argmax_out != nullptr || cur.argmax_out != nullptr) return false;
-  const Span pw[3] = {span_of(prev.out0, M, prev.ld_out, prev.N, 2), span_of(prev.out1, M, prev.ld_out, prev.N, 2),
-                      span_of(prev.xout, M, prev.ld_xout, prev.K, 2)};
-  const Span pr[2] = {span_of(prev.in0, M, prev.ld_in, prev.K, 2), span_of(prev.in1, M, prev.ld_in, prev.K, 2)};
-  const Span cw[2] = {span_of(cur.out0, M, cur.ld_out, cur.N, 2), span_of(cur.out1, M, cur.ld_out, cur.N, 2)};
-  const Span cr[1] = {span_of(cur.in0, M, cur.ld_in, cur.K, 2)};
+  const Span pw[3] = {span_of(prev.out0, prev.rows, prev.ld_out, prev.N, 2), span_of(prev.out1, prev.rows, prev.ld_out, prev.N, 2),
+                      span_of(prev.xout, prev.rows, prev.ld_xout, prev.K, 2)};
+  const Span pr[2] = {span_of(prev.in0, prev.rows, prev.ld_in, prev.K, 2), span_of(prev.in1, prev.rows, prev.ld_in, prev.K, 2)};
+  const Span cw[2] = {span_of(cur.out0, cur.rows, cur.ld_out, cur.N, 2), span_of(cur.out1, cur.rows, cur.ld_out, cur.N, 2)};
+  const Span cr[1] = {span_of(cur.in0, cur.rows, cur.ld_in, cur.K, 2)};
   for (const Span& a : cw) {
     for (const Span& b : pw) if (overlap(a, b)) return false;
     for (const Span& b : pr) if (overlap(a, b)) return false;
@@ -199,13 +200,13 @@ static bool independent_ops(const MegaOp& prev, const MegaOp& cur, int M) {
 
 // True if the run is a list of plain linears no two of which share a buffer other than inputs
 // that both only read: nothing in it has to wait for a result.
-static bool independent_run(const std::vector<MegaOp>& mega, int M) {
+static bool independent_run(const std::vector<MegaOp>& mega) {
   if (mega.size() < 2) return false;
   for (const MegaOp& m : mega)
     if (m.packed1 != nullptr || m.prologue != 0 || m.emit_ssq != 0 || m.argmax_out != nullptr || m.out0 == nullptr) return false;
   for (size_t a = 0; a < mega.size(); ++a)
     for (size_t b = a + 1; b < mega.size(); ++b)
-      if (!independent_ops(mega[a], mega[b], M) || !independent_ops(mega[b], mega[a], M)) return false;
+      if (!independent_ops(mega[a], mega[b]) || !independent_ops(mega[b], mega[a])) return false;
   return true;
 }
 
@@ -271,7 +272,7 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
       // Independent plain linears form ONE run: their chunks are laid end to end and every CTA
       // takes one contiguous piece.  Anything else is a chain: every operation is its own run and
       // waits for the one before it.
-      const bool indep = independent_run(mega, run_M);
+      const bool indep = independent_run(mega);
       const bool batch = indep;
       bool x_ring = false;
       if (batch) {
@@ -332,6 +333,55 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
     }
     return QL_OK;
   };
+
+  // A list of plain linears with one common row count above 16: every linear becomes ceil(M / 16)
+  // operations of at most 16 rows each (the persistent kernel's row count), which write disjoint rows
+  // and therefore form one stream together with the other linears' slabs.  The weights are then
+  // unpacked once per slab, but cross HBM about once: the slabs of a linear are neighbours in the
+  // stream, so thread blocks work on them at the same time and meet in L2.
+  bool slabs = n_ops > 0;
+  for (int i = 0; i < n_ops && slabs; ++i) {
+    const ql_op& o = ops[i];
+    slabs = o.kind == QL_OP_LINEAR && o.M > 16 && o.M == ops[0].M && o.g == ops[0].g && o.argmax_out == nullptr &&
+            o.out != nullptr && o.draft_ids == nullptr && ws_total_bytes(o.N / kTileN, 16) <= workspace_bytes;
+    if (slabs) {
+      ql_op probe_op = o;
+      probe_op.M = 16;
+      MegaOp probe = make_mega(probe_op, nullptr);
+      run_split(probe.total_chunks, (uint32_t)stack_ncta(sms), probe.nc, probe.cq, probe.cr);
+      slabs = stack_plan(&probe, 1, o.g, sms).ok;
+    }
+  }
+  if (slabs) {
+    static thread_local std::vector<MegaOp> all;
+    all.clear();
+    for (int i = 0; i < n_ops; ++i) {
+      for (int r0 = 0; r0 < ops[i].M; r0 += 16) {
+        ql_op so = ops[i];
+        so.M = ops[i].M - r0 < 16 ? ops[i].M - r0 : 16;
+        so.in0 = ops[i].in0 + (size_t)r0 * ops[i].ld_in;
+        so.out = ops[i].out + (size_t)r0 * ops[i].ld_out;
+        all.push_back(make_mega(so, nullptr));
+      }
+    }
+    // only a stream of independent operations gains from this; linears that depend on one another
+    // keep their one launch each
+    if (independent_run(all)) {
+      run_M = 16;
+      run_g = ops[0].g;
+      for (const MegaOp& m : all) {
+        if ((int)mega.size() >= kStackRunOps) {
+          const int st = flush();
+          if (st != QL_OK) return st;
+        }
+        mega.push_back(m);
+      }
+      const int st = flush();
+      if (dry != nullptr) *dry = cnt;
+      if (counts_out != nullptr) *counts_out = cnt;
+      return st;
+    }
+  }
 
   for (int i = 0; i < n_ops; ++i) {
     const ql_op& o = ops[i];

@@ -60,14 +60,16 @@ struct MegaOp {
   int emit_ssq;            // 0: none; 1: per-tile row sums of bf16(Y)^2; 2: of (silu(bf16 Y0) * bf16 Y1)^2
   const int32_t* draft_ids;  // [M] drafted tokens the greedy tokens are compared with (verification tail), else nullptr
   int32_t* accept_out;       // [2] accepted-prefix length, bonus token
-  uint64_t pad_[2];
+  int rows;                  // rows of X and Y this operation works on (1..16)
+  int pad0_;
+  uint64_t pad_;
 };
 static_assert(sizeof(MegaOp) == kOpDescBytes, "operation descriptor layout");
 
 struct StackParams {
   const MegaOp* ops;       // device copy of the descriptors (in the workspace)
   int n_ops;
-  int M;
+  int M;                   // (host bookkeeping; the kernel takes the row count of every operation from its descriptor)
   int ncta;
   int n_stages;            // ring depth
   int n_x;                 // X slots (groups) in shared memory

@@ -216,6 +216,7 @@ __device__ __forceinline__ void build_x(const StackParams& sp, const MegaOp& d, 
   const uint32_t g_first = start % Gn;
   const uint32_t n_units = n_x * UPG;
   const int prologue = d.prologue;
+  const int rows = d.rows;
   const int ld_in = d.ld_in;
   const uint16_t* in0 = d.in0;
   // unit idx: slot k = idx / UPG, row m = (idx / UPR) % MP, k-unit ku = idx % UPR: lanes run along K
@@ -238,7 +239,7 @@ __device__ __forceinline__ void build_x(const StackParams& sp, const MegaOp& d, 
   } else if (prologue == 0) {
     for (uint32_t idx = tid; idx < n_units; idx += kUnpackThreads) {
       const uint32_t m = unit_row(idx);
-      const bool live = (int)m < sp.M;
+      const bool live = (int)m < rows;
       cp_async16(unit_addr(idx), live ? (in0 + (size_t)m * ld_in + unit_col(idx)) : in0, live ? 16u : 0u);
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
@@ -250,7 +251,7 @@ __device__ __forceinline__ void build_x(const StackParams& sp, const MegaOp& d, 
     auto emit = [&](uint32_t idx, uint4 o) {
       const uint32_t m = unit_row(idx);
       // the CTA that owns (tile 0, group Gi) writes the normalised X out for the record
-      if (xout != nullptr && (int)m < sp.M && start + idx / UPG < Gn)
+      if (xout != nullptr && (int)m < rows && start + idx / UPG < Gn)
         *reinterpret_cast<uint4*>(xout + (size_t)m * ld_xout + unit_col(idx)) = o;
       *reinterpret_cast<uint4*>(unit_addr(idx)) = o;
     };
@@ -270,7 +271,7 @@ __device__ __forceinline__ void build_x(const StackParams& sp, const MegaOp& d, 
         for (int q = 0; q < XB; ++q) {
           const uint32_t idx = base + q * kUnpackThreads;
           ra[q] = make_uint4(0u, 0u, 0u, 0u);
-          if (idx < n_units && (int)unit_row(idx) < sp.M)
+          if (idx < n_units && (int)unit_row(idx) < rows)
             ra[q] = __ldcg(reinterpret_cast<const uint4*>(in0 + (size_t)unit_row(idx) * ld_in + unit_col(idx)));
         }
         need_inv();
@@ -278,7 +279,7 @@ __device__ __forceinline__ void build_x(const StackParams& sp, const MegaOp& d, 
         for (int q = 0; q < XB; ++q) {
           const uint32_t idx = base + q * kUnpackThreads;
           if (idx >= n_units) continue;
-          const float inv = (int)unit_row(idx) < sp.M ? s_inv[unit_row(idx)] : 0.f;
+          const float inv = (int)unit_row(idx) < rows ? s_inv[unit_row(idx)] : 0.f;
           uint4 o;
           o.x = pack_bf16x2_rn(bf16lo_to_f32(ra[q].x) * inv, bf16hi_to_f32(ra[q].x) * inv);
           o.y = pack_bf16x2_rn(bf16lo_to_f32(ra[q].y) * inv, bf16hi_to_f32(ra[q].y) * inv);
@@ -297,7 +298,7 @@ __device__ __forceinline__ void build_x(const StackParams& sp, const MegaOp& d, 
         for (int q = 0; q < XB; ++q) {
           const uint32_t idx = base + q * kUnpackThreads;
           ra[q] = make_uint4(0u, 0u, 0u, 0u); rb[q] = ra[q];
-          if (idx < n_units && (int)unit_row(idx) < sp.M) {
+          if (idx < n_units && (int)unit_row(idx) < rows) {
             const uint4* p = reinterpret_cast<const uint4*>(act + (size_t)unit_row(idx) * K + unit_col(idx));
             ra[q] = __ldcg(p);
             rb[q] = __ldcg(p + 1);
@@ -308,7 +309,7 @@ __device__ __forceinline__ void build_x(const StackParams& sp, const MegaOp& d, 
         for (int q = 0; q < XB; ++q) {
           const uint32_t idx = base + q * kUnpackThreads;
           if (idx >= n_units) continue;
-          const float inv = (int)unit_row(idx) < sp.M ? s_inv[unit_row(idx)] : 0.f;
+          const float inv = (int)unit_row(idx) < rows ? s_inv[unit_row(idx)] : 0.f;
           uint4 o;
           o.x = pack_bf16x2_rn(__uint_as_float(ra[q].x) * inv, __uint_as_float(ra[q].y) * inv);
           o.y = pack_bf16x2_rn(__uint_as_float(ra[q].z) * inv, __uint_as_float(ra[q].w) * inv);
@@ -527,6 +528,7 @@ __global__ void __launch_bounds__(RING ? kStThreadsRing : kStThreads, 1) qstack_
         if (start >= end) continue;
         const uint16_t* in0 = ldg_ptr(&ops[j].in0);
         const int ld_in = __ldg(&ops[j].ld_in);
+        const int rows = __ldg(&ops[j].rows);
         const uint32_t Gn = (uint32_t)h.n_groups;
         for (uint32_t c = start; c < end; ++c, ++r) {
           const uint32_t slot = r % P;
@@ -541,7 +543,7 @@ __global__ void __launch_bounds__(RING ? kStThreadsRing : kStThreads, 1) qstack_
 #pragma unroll
           for (uint32_t u = (uint32_t)lane; u < (uint32_t)MP * UPR; u += 32) {
             const uint32_t m = u / UPR, ku = u % UPR;
-            const bool live = (int)m < sp.M;
+            const bool live = (int)m < rows;
             cp_async16(dst + ku * kXLbo + (m >> 3) * 128u + (m & 7u) * 16u,
                        live ? (in0 + (size_t)m * ld_in + (size_t)Gi * G + ku * 8) : in0, live ? 16u : 0u);
           }
@@ -870,7 +872,8 @@ __global__ void __launch_bounds__(RING ? kStThreadsRing : kStThreads, 1) qstack_
           const int emit_ssq = dsc.emit_ssq;
           const int ld_out = dsc.ld_out;
           const int col = (int)T * kTileN + 4 * lane;
-          const bool live = rw < sp.M;
+          const int op_rows = dsc.rows;
+          const bool live = rw < op_rows;
           float a[4];
           uint2 y0;
           y0.x = pack_bf16x2_rn(f0[0], f0[1]);
@@ -955,18 +958,18 @@ __global__ void __launch_bounds__(RING ? kStThreadsRing : kStThreads, 1) qstack_
                 if (lane == 0) {
                   fence_gpu();                           // release: this row's token
                   asm volatile("atom.add.relaxed.gpu.global.s32 %0, [%1], 1;" : "=r"(rows_done) : "l"(amax_cnt + 16 * 32) : "memory");
-                  if (rows_done == sp.M - 1) fence_gpu();   // acquire: the other rows' tokens
+                  if (rows_done == op_rows - 1) fence_gpu();   // acquire: the other rows' tokens
                 }
                 rows_done = __shfl_sync(0xffffffffu, rows_done, 0);
-                if (rows_done == sp.M - 1) {
-                  const int tok = lane < sp.M ? (lane == rw ? bi : __ldcg(&argmax_out[lane])) : -1;
-                  const int drf = lane < sp.M ? __ldg(&dsc.draft_ids[lane]) : -2;
-                  const unsigned agree = __ballot_sync(0xffffffffu, lane < sp.M && tok == drf);
+                if (rows_done == op_rows - 1) {
+                  const int tok = lane < op_rows ? (lane == rw ? bi : __ldcg(&argmax_out[lane])) : -1;
+                  const int drf = lane < op_rows ? __ldg(&dsc.draft_ids[lane]) : -2;
+                  const unsigned agree = __ballot_sync(0xffffffffu, lane < op_rows && tok == drf);
                   const int a = __ffs(~agree) - 1;            // first row that disagrees (rows >= M never agree)
-                  const int bonus = __shfl_sync(0xffffffffu, tok, a < sp.M ? a : 0);
+                  const int bonus = __shfl_sync(0xffffffffu, tok, a < op_rows ? a : 0);
                   if (lane == 0) {
                     dsc.accept_out[0] = a;
-                    dsc.accept_out[1] = a < sp.M ? bonus : -1;
+                    dsc.accept_out[1] = a < op_rows ? bonus : -1;
                     amax_cnt[16 * 32] = 0;
                   }
                 }

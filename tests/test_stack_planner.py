@@ -86,6 +86,19 @@ def test_independent_linears_skip_the_wait_but_write_after_write_does_not(ql):
     assert plan(ql, [a, b])["independent"] == 0
 
 
+def test_lists_of_plain_linears_above_16_rows_become_slabs(ql):
+    def big(i, M, out=None):
+        return dict(kind=0, M=M, K=2560, N=2560, g=128, ld_in=2560, ld_out=2560, packed=buf(100 + i), in0=buf(1), out=buf(20 + i) if out is None else out)
+    c = plan(ql, [big(i, 64) for i in range(3)], M=64)
+    assert c["stack_launches"] == 1 and c["fused_ops"] == 12 and c["batch_launches"] == 1 and c["single_linears"] == 0
+    c = plan(ql, [big(i, 40) for i in range(2)], M=64)
+    assert c["fused_ops"] == 6 and c["batch_launches"] == 1                      # 16 + 16 + 8 rows
+    c = plan(ql, [big(0, 32), big(1, 48)], M=64)                                  # different row counts: one launch each
+    assert c["stack_launches"] == 0 and c["single_linears"] == 2
+    c = plan(ql, [big(0, 32, out=buf(20)), big(1, 32, out=buf(20))], M=64)        # same output: ordered, one launch each
+    assert c["stack_launches"] == 0 and c["single_linears"] == 2
+
+
 def test_m_above_16_and_mixed_group_sizes(ql):
     big = dict(kind=0, M=32, K=2560, N=2560, g=128, ld_in=2560, ld_out=2560, packed=buf(100), in0=buf(1), out=buf(2))
     c = plan(ql, [big, big], M=32)
