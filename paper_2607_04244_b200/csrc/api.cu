@@ -297,7 +297,7 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
       StackParams sp = {};
       sp.ws = ws_carve(workspace, n_tiles_cap, 16);
       sp.ops = reinterpret_cast<const MegaOp*>(sp.ws.desc);
-      sp.n_ops = (int)mega.size(); sp.M = run_M; sp.ncta = plan.ncta; sp.n_stages = plan.n_stages; sp.n_x = plan.n_x; sp.x_ring = plan.x_ring;
+      sp.n_ops = (int)mega.size(); sp.M = run_M; sp.ncta = plan.ncta; sp.n_stages = plan.n_stages; sp.n_x = plan.n_x; sp.x_ring = plan.x_ring; sp.one_stream = batch ? 1 : 0;
       sp.wait_ns = g_wait_ns.load(std::memory_order_relaxed);
       sp.ablate = g_ablate.load(std::memory_order_relaxed);
       sp.timeline = g_timeline.load(std::memory_order_relaxed);

@@ -75,6 +75,7 @@ struct StackParams {
   int n_x;                 // X slots (groups) in shared memory
   int x_ring;              // 0: X of an operation is built once, by the unpack threads; P > 0 (one stream of independent
                            // linears): the X slots are a ring of P chunks filled by a loader warp, chunk by chunk
+  int one_stream;          // the operations are independent plain linears laid end to end (selects the kernel variant)
   int ablate;              // timing experiments only (see the stack kernel); 0 in production
   uint32_t epoch;          // launch number: partial tiles in the workspace carry (epoch, operation) tags
   uint64_t wait_ns;        // budget of every bounded wait

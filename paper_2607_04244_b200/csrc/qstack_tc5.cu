@@ -11,8 +11,10 @@
 //   16     producer: one bulk copy (TMA engine, no tensor map, no multicast) per packed chunk into a
 //          ring of shared-memory stages; it runs ahead over operation boundaries, so the weights of
 //          operation j+1 are on chip while operation j is still being reduced.
-//   17-20  one MMA issuer per unpack group (a tcgen05.mma with N = 16 costs its issuing thread
-//          ~150 cycles while tensor-memory stores are running, and a chunk needs 8).
+//   17-20  one MMA-issuing thread per unpack group (a tcgen05.mma with N = 16 costs its issuing thread
+//          ~100 cycles while tensor-memory stores are running, and a chunk needs 8); in the variant
+//          for chains two of them share a warp (lanes 0 and 16), so that 20 warps leave 96 registers
+//          per thread; the watcher and the X loader follow the issuer warps.
 //   21     watcher: polls the counter of the previous operation, so that the other warps can work
 //          while they wait, and computes the row scales 1/rms from the per-tile sums of squares.
 //   22     X loader, only for one stream of independent linears: copies the X columns of every chunk
@@ -47,11 +49,13 @@ constexpr int NWG = 4;                                  // unpack groups per CTA
 constexpr int AH = 3;                                   // half-chunk A buffers per group
 constexpr int MP = 16;                                  // padded rows
 constexpr int kUnpackThreads = NWG * 128;               // 512
-constexpr int kIssuers = NWG;                           // one per group
-constexpr int kWarpProducer = NWG * 4, kWarpIssuer0 = NWG * 4 + 1, kWarpWatcher = NWG * 4 + 1 + kIssuers;
-constexpr int kWarpXLoader = kWarpWatcher + 1;           // exists only in the kernel variant with the X ring
-constexpr int kStThreads = (kWarpWatcher + 1) * 32;     // 704
-constexpr int kStThreadsRing = (kWarpXLoader + 1) * 32; // 736
+constexpr int kWarpProducer = NWG * 4, kWarpIssuer0 = NWG * 4 + 1;
+// One issuing thread per unpack group.  PAIRED (chains): two of them share a warp (lanes 0 and 16), the CTA has
+// 20 warps and 96 registers per thread - in a chain the issuers mostly wait, and the unpack loop gains more
+// from the registers than it loses from the shared issue slot.  Streams keep one warp per issuer (80 registers).
+__host__ __device__ constexpr int st_issuer_warps(bool paired) { return paired ? NWG / 2 : NWG; }
+__host__ __device__ constexpr int st_warp_watcher(bool paired) { return kWarpIssuer0 + st_issuer_warps(paired); }
+__host__ __device__ constexpr int st_threads(bool ring, bool paired) { return (st_warp_watcher(paired) + 1 + (ring ? 1 : 0)) * 32; }   // the X loader follows the watcher
 constexpr int kXRingSlots = 16;                         // X slots of the ring (one stream of independent linears)
 constexpr int kStMaxStages = 24;
 constexpr uint32_t kStSmemBudget = 232448u;
@@ -327,8 +331,10 @@ __device__ __forceinline__ void build_x(const StackParams& sp, const MegaOp& d, 
 
 // RING: variant for one stream of independent linears whose X does not fit per operation (one more
 // warp, the X loader; the issuers take X slot by slot).  The other variant has none of that code.
-template <int G, bool RING>
-__global__ void __launch_bounds__(RING ? kStThreadsRing : kStThreads, 1) qstack_tc5_kernel(const __grid_constant__ StackParams sp) {
+template <int G, bool RING, bool PAIRED>
+__global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel(const __grid_constant__ StackParams sp) {
+  constexpr int kWarpWatcher = st_warp_watcher(PAIRED);
+  constexpr int kWarpXLoader = kWarpWatcher + 1;
   extern __shared__ __align__(1024) uint8_t smem[];
   constexpr uint32_t STAGE = align128(chunk_bytes(G));
   constexpr uint32_t XSLOT = st_xslot_bytes(G);
@@ -393,7 +399,7 @@ __global__ void __launch_bounds__(RING ? kStThreadsRing : kStThreads, 1) qstack_
     tmem_alloc(s_tmem, TMEM_COLS);
     tmem_relinquish();
   }
-  for (int i = tid; i < 2 * sp.n_ops; i += (RING ? kStThreadsRing : kStThreads))
+  for (int i = tid; i < 2 * sp.n_ops; i += st_threads(RING, PAIRED))
     s_heads[i] = __ldg(reinterpret_cast<const uint4*>(ops + (i >> 1)) + (i & 1));
   tc_fence_before_sync();
   __syncthreads();
@@ -555,9 +561,9 @@ __global__ void __launch_bounds__(RING ? kStThreadsRing : kStThreads, 1) qstack_
     }
   } else if (warp >= kWarpIssuer0) {
     // ------------------------------------------------------------------ MMA issue for unpack group w
-    if (lane == 0) {
+    if (PAIRED ? (lane & 15) == 0 : lane == 0) {
       constexpr uint32_t idesc = tc_idesc_bf16_m128(MP);
-      const uint32_t w = warp - kWarpIssuer0;             // unpack group served
+      const uint32_t w = PAIRED ? 2 * (warp - kWarpIssuer0) + (lane >> 4) : warp - kWarpIssuer0;   // unpack group served
       const uint64_t desc0 = tc_smem_desc_kmajor(smem_u32(xbuf), kXLbo, 128u);
       constexpr uint32_t KSTEP = (2u * kXLbo) >> 4;     // one MMA contracts 16 rows of K = two core matrices
       constexpr uint32_t SLOT = XSLOT >> 4;
@@ -1066,19 +1072,21 @@ StackPlan stack_plan(const MegaOp* ops, int n_ops, int g, int sms, bool one_stre
   return r;
 }
 
-template <int G, bool RING>
+template <int G, bool RING, bool PAIRED>
 static cudaError_t stack_launch_g(const StackParams& sp, size_t smem, cudaStream_t stream) {
   // all CTAs wait on one another's progress: they must be co-resident (the cooperative launch checks it)
-  cudaError_t e = cudaFuncSetAttribute(qstack_tc5_kernel<G, RING>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStSmemBudget);
+  cudaError_t e = cudaFuncSetAttribute(qstack_tc5_kernel<G, RING, PAIRED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStSmemBudget);
   if (e != cudaSuccess) return e;
   void* args[] = {const_cast<StackParams*>(&sp)};
-  return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(qstack_tc5_kernel<G, RING>), dim3(sp.ncta),
-                                     dim3(RING ? kStThreadsRing : kStThreads), args, smem, stream);
+  return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(qstack_tc5_kernel<G, RING, PAIRED>), dim3(sp.ncta),
+                                     dim3(st_threads(RING, PAIRED)), args, smem, stream);
 }
 
+// Three variants: chains (paired issuers), one stream with X resident per operation, one stream with the X ring.
 cudaError_t launch_stack_tc5(const StackParams& sp, int g, size_t smem, cudaStream_t stream) {
-  if (sp.x_ring > 0) return g == 128 ? stack_launch_g<128, true>(sp, smem, stream) : stack_launch_g<64, true>(sp, smem, stream);
-  return g == 128 ? stack_launch_g<128, false>(sp, smem, stream) : stack_launch_g<64, false>(sp, smem, stream);
+  if (sp.x_ring > 0) return g == 128 ? stack_launch_g<128, true, false>(sp, smem, stream) : stack_launch_g<64, true, false>(sp, smem, stream);
+  if (sp.one_stream) return g == 128 ? stack_launch_g<128, false, false>(sp, smem, stream) : stack_launch_g<64, false, false>(sp, smem, stream);
+  return g == 128 ? stack_launch_g<128, false, true>(sp, smem, stream) : stack_launch_g<64, false, true>(sp, smem, stream);
 }
 
 }  // namespace ql
