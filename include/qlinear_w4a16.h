@@ -324,6 +324,19 @@ int ql_attn_plan(int n_q, int T, int Hq, int Hkv, int d, int p0, int window, int
 uint32_t ql_plan_first_chunk(uint32_t total_chunks, uint32_t ncta, uint32_t cta);
 uint32_t ql_plan_chunk_owner(uint32_t total_chunks, uint32_t ncta, uint32_t chunk);
 
+/* The split a CHAINED operation of n_tiles column tiles (a gate/up pair counts its double tiles)
+ * and n_groups quantisation groups gets on ncta thread blocks (host copy of what the kernel
+ * resolves, for tests).  range[0..1] = the chunks [lo, hi) of thread block `cta` (chunk
+ * T * n_groups + G is group G of tile T); range[2] = 1 for the aligned split (at most ncta / 2 tiles
+ * and at least two chunks per thread block: every tile has thread blocks of its own, and the first
+ * of them, which adds the others' partial rows and finishes the tile, has `owner extra` chunks more
+ * than an even share of the rest), 0 for the even stream-K split; range[3] = the last thread block
+ * that works on the tile of chunk hi - 1.  Returns QL_OK, QL_ERR_NULL or QL_ERR_SHAPE.
+ * ql_debug_set_owner_extra(e): measurement hook, process-wide, for the calls that follow: the
+ * owner's extra chunks (-1: the default of 4; below -1: even split everywhere). */
+int ql_plan_chain_split(int n_tiles, int n_groups, int ncta, int cta, uint32_t range[4]);
+void ql_debug_set_owner_extra(int chunks);
+
 /* Test hooks for the bounded waits of the persistent kernel (process-wide; not for production use).
  * ql_debug_set_wait_budget_ns: budget of every wait inside qlinear_stack_w4a16 launches that
  * follow (0 restores the default of 2 s).  ql_debug_no_release(i): in the launches that follow, the

@@ -24,6 +24,7 @@ EXPORTS = [
     "ql_device_status_raw",
     "qpack_w4_g128", "qrequant_pack_w4", "qlinear_w4a16", "qlinear_w4a16_path", "ql_select_path", "qlinear_stack_w4a16",
     "qlinear_stack_w4a16_host", "ql_launch_count", "qlinear_w4a16_static", "ql_static_status", "ql_stack_plan", "ql_linear_plan", "ql_plan_first_chunk", "ql_plan_chunk_owner",
+    "ql_plan_chain_split", "ql_debug_set_owner_extra",
     "ql_attn_workspace_bytes", "qattn_swa_bf16", "ql_attn_plan",
     "ql_debug_set_wait_budget_ns", "ql_debug_no_release", "ql_debug_set_timeline", "ql_debug_timeline_enabled", "ql_debug_set_ablate",
 ]
@@ -103,6 +104,10 @@ def load(path: str | None = None):
     for fn in (lib.ql_plan_first_chunk, lib.ql_plan_chunk_owner):
         fn.restype = ctypes.c_uint32
         fn.argtypes = [ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32]
+    lib.ql_plan_chain_split.restype = i32
+    lib.ql_plan_chain_split.argtypes = [i32, i32, i32, i32, ctypes.POINTER(ctypes.c_uint32)]
+    lib.ql_debug_set_owner_extra.restype = None
+    lib.ql_debug_set_owner_extra.argtypes = [i32]
     lib.ql_debug_set_wait_budget_ns.restype = None
     lib.ql_debug_set_wait_budget_ns.argtypes = [ctypes.c_uint64]
     lib.ql_debug_no_release.restype = None
@@ -154,6 +159,18 @@ def ql_launch_count() -> int:
 
 def ql_debug_set_wait_budget_ns(ns: int) -> None:
     load().ql_debug_set_wait_budget_ns(ns)
+
+
+def ql_plan_chain_split(n_tiles: int, n_groups: int, ncta: int, cta: int) -> dict:
+    """The chunks [lo, hi) thread block `cta` gets of a chained operation, whether the split is the
+    aligned one, and the last thread block of the tile of chunk hi - 1."""
+    r = (ctypes.c_uint32 * 4)()
+    _check(load().ql_plan_chain_split(n_tiles, n_groups, ncta, cta, r), "ql_plan_chain_split")
+    return {"lo": int(r[0]), "hi": int(r[1]), "aligned": bool(r[2]), "last_cta": int(r[3])}
+
+
+def ql_debug_set_owner_extra(chunks: int = -1) -> None:
+    load().ql_debug_set_owner_extra(chunks)
 
 
 def ql_debug_no_release(fused_op: int) -> None:

@@ -29,6 +29,8 @@ static std::atomic<uint64_t> g_wait_ns{kWaitBudgetNs};    // budget of the stack
 // debug hook changes: a remembered plan is valid only while nothing of that happened since it was staged.
 static std::atomic<uint64_t> g_desc_gen{1};
 static std::atomic<int> g_no_release_op{-1};              // test hook: fused operation that does not publish its tiles
+constexpr int kOwnerExtraChunks = 4;                      // aligned split: chunks the owner of a tile takes beyond an even share
+static std::atomic<int> g_owner_extra{kOwnerExtraChunks}; // (measurement hook ql_debug_set_owner_extra; negative: even split everywhere)
 static std::atomic<int> g_ablate{0};                      // timing experiments: phases of the stack kernel switched off
 static std::atomic<uint64_t*> g_timeline{nullptr};        // device buffer for the in-kernel timeline (QL_TIMELINE builds)
 
@@ -217,6 +219,26 @@ static void split_one_stream(std::vector<MegaOp>& mega, int ncta) {
   for (MegaOp& m : mega) run_split(total, (uint32_t)ncta, m.nc, m.cq, m.cr);
 }
 
+// Split of a chained operation.  Where every tile can have at least two CTAs of its own and two
+// chunks for each of them (the fused qkv, attention-output and MLP-down projections of a verify
+// step: 48 or 20 tiles on 148 CTAs), the aligned split is taken: no CTA meets two tiles, and the
+// first CTA of a tile - its owner, which has to wait for the others' partial rows before it can
+// finish the tile - unpacks g_owner_extra chunks more than they do in the meantime.  Otherwise
+// (gate/up pairs: 76 double tiles; the LM head) the chunks are shared out evenly and pieces cross
+// tile boundaries.
+static void chain_split(MegaOp& m, int ncta) {
+  m.cat_base = 0;
+  const uint32_t nt = (uint32_t)m.n_tiles, Gn = (uint32_t)m.n_groups, nc = (uint32_t)ncta;
+  const uint32_t most = (nc + nt - 1) / nt;                  // CTAs of the best-served tile
+  const int extra_want = g_owner_extra.load(std::memory_order_relaxed);
+  if (extra_want >= 0 && 2 * nt <= nc && Gn >= 2 * most) {
+    const uint32_t extra = (uint32_t)extra_want < Gn - most ? (uint32_t)extra_want : Gn - most;   // everyone keeps at least one chunk
+    m.nc = nc; m.cq = extra; m.cr = kSplitAligned | nt;
+    return;
+  }
+  run_split(m.total_chunks, nc, m.nc, m.cq, m.cr);
+}
+
 static bool is_dual(const ql_op* ops, int i, int n_ops) {
   if (i + 2 >= n_ops) return false;
   const ql_op &a = ops[i], &b = ops[i + 1], &c = ops[i + 2];
@@ -283,8 +305,7 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
       } else {
         for (size_t j = 0; j < mega.size(); ++j) {
           MegaOp& m = mega[j];
-          m.cat_base = 0;
-          run_split(m.total_chunks, (uint32_t)ncta, m.nc, m.cq, m.cr);
+          chain_split(m, ncta);
           if (j > 0) m.flags |= kOpWait;
         }
       }
@@ -395,7 +416,7 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
       bool fits = o.M <= 16 && ws_total_bytes(m.n_tiles, 16) <= workspace_bytes;
       if (fits) {
         MegaOp probe = m;                               // would it fit as a chained operation?
-        run_split(probe.total_chunks, (uint32_t)stack_ncta(sms), probe.nc, probe.cq, probe.cr);
+        chain_split(probe, stack_ncta(sms));
         fits = stack_plan(&probe, 1, o.g, sms).ok;
       }
       if (fits && !mega.empty() && (o.M != run_M || o.g != run_g)) {
@@ -776,6 +797,19 @@ uint32_t ql_plan_chunk_owner(uint32_t total_chunks, uint32_t ncta, uint32_t chun
   return run_chunk_owner(nc, cq, cr, chunk);
 }
 
+int ql_plan_chain_split(int n_tiles, int n_groups, int ncta, int cta, uint32_t range[4]) {
+  if (range == nullptr) return QL_ERR_NULL;
+  if (n_tiles < 1 || n_groups < 1 || ncta < 1 || ncta > kMaxCtas / 2 || cta < 0 || cta >= ncta) return QL_ERR_SHAPE;
+  MegaOp m = {};
+  m.n_tiles = n_tiles; m.n_groups = n_groups;
+  m.total_chunks = (uint32_t)n_tiles * (uint32_t)n_groups;
+  chain_split(m, ncta);
+  op_local_range(m.nc, m.cq, m.cr, 0, m.total_chunks, (uint32_t)cta, range[0], range[1]);
+  range[2] = (m.cr & kSplitAligned) ? 1u : 0u;
+  range[3] = range[0] < range[1] ? op_last_cta(m.nc, m.cq, m.cr, 0, (uint32_t)n_groups, (range[1] - 1) / (uint32_t)n_groups) : 0u;
+  return QL_OK;
+}
+
 void ql_debug_set_wait_budget_ns(uint64_t ns) { g_desc_gen.fetch_add(1, std::memory_order_relaxed); g_wait_ns.store(ns == 0 ? kWaitBudgetNs : ns, std::memory_order_relaxed); }
 void ql_debug_set_timeline(void* device_buffer) { g_desc_gen.fetch_add(1, std::memory_order_relaxed); g_timeline.store(static_cast<uint64_t*>(device_buffer), std::memory_order_relaxed); }
 int ql_debug_timeline_enabled(void) {
@@ -786,6 +820,10 @@ int ql_debug_timeline_enabled(void) {
 #endif
 }
 void ql_debug_set_ablate(int mask) { g_desc_gen.fetch_add(1, std::memory_order_relaxed); g_ablate.store(mask, std::memory_order_relaxed); }
+void ql_debug_set_owner_extra(int chunks) {
+  g_desc_gen.fetch_add(1, std::memory_order_relaxed);
+  g_owner_extra.store(chunks == -1 ? kOwnerExtraChunks : chunks, std::memory_order_relaxed);
+}
 void ql_debug_no_release(int fused_op) { g_desc_gen.fetch_add(1, std::memory_order_relaxed); g_no_release_op.store(fused_op, std::memory_order_relaxed); }
 
 uint64_t ql_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

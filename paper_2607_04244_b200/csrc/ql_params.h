@@ -40,7 +40,8 @@ constexpr int kOpLazy = 16;       // nothing in the launch waits for this operat
                                   // next tile segment may be started before the current one is finished
 constexpr int kOpNoRelease = 4;   // test hook: finished tiles are not published (the next operation's wait runs out)
 struct MegaOp {
-  uint32_t nc, cq, cr;     // CTA i owns run positions [i*cq + i*cr/nc, (i+1)*cq + (i+1)*cr/nc), i < nc
+  uint32_t nc, cq, cr;     // CTA i owns run positions [i*cq + i*cr/nc, (i+1)*cq + (i+1)*cr/nc), i < nc; or, with
+                           // cr = kSplitAligned | n_tiles and cq = the owner's extra chunks, the aligned split
   uint32_t cat_base;       // run position of this operation's chunk 0
   uint32_t total_chunks;   // n_tiles * n_groups (per matrix)
   int n_groups, n_tiles;
@@ -87,11 +88,32 @@ struct StackParams {
 __host__ __device__ inline uint32_t run_first_chunk(uint32_t nc, uint32_t cq, uint32_t cr, uint32_t i) {
   return i * cq + (i * cr) / nc;
 }
+// Aligned split of a chained operation with at most nc / 2 tiles (cr = kSplitAligned | n_tiles, cq = the
+// owner's extra chunks e): tile T belongs to the CTAs [T nc / n_tiles, (T + 1) nc / n_tiles) alone, so no CTA
+// works on two tiles and nobody ends a tile segment in the middle of its piece.  The first CTA of a tile
+// (its owner: it adds the others' partial rows and finishes the tile) takes e chunks more than an even
+// share of the rest: that is the time the others' partial rows need to reach it.
+constexpr uint32_t kSplitAligned = 0x80000000u;
+__host__ __device__ inline void aligned_tile_ctas(uint32_t nc, uint32_t nt, uint32_t T, uint32_t& c0, uint32_t& c1) {
+  c0 = (T * nc) / nt;
+  c1 = ((T + 1) * nc) / nt;
+}
+__host__ __device__ inline void aligned_range(uint32_t nc, uint32_t extra, uint32_t nt, uint32_t total, uint32_t i,
+                                              uint32_t& lo, uint32_t& hi) {
+  const uint32_t Gn = total / nt;
+  const uint32_t T = ((i + 1) * nt + nc - 1) / nc - 1;   // the largest T with T nc / nt <= i
+  uint32_t c0, c1;
+  aligned_tile_ctas(nc, nt, T, c0, c1);
+  const uint32_t n = c1 - c0, r = i - c0, rest = Gn - extra;
+  lo = T * Gn + (r == 0 ? 0u : extra + (r * rest) / n);
+  hi = T * Gn + extra + ((r + 1) * rest) / n;
+}
 // Chunks [lo, hi) of operation `op` (per matrix) that CTA i owns; lo == hi if none.
 __host__ __device__ inline void op_local_range(uint32_t nc, uint32_t cq, uint32_t cr, uint32_t cat_base, uint32_t total,
                                                uint32_t i, uint32_t& lo, uint32_t& hi) {
   lo = hi = 0;
   if (i >= nc) return;
+  if (cr & kSplitAligned) { aligned_range(nc, cq, cr & ~kSplitAligned, total, i, lo, hi); return; }
   uint32_t a = run_first_chunk(nc, cq, cr, i), b = run_first_chunk(nc, cq, cr, i + 1);
   const uint32_t top = cat_base + total;
   if (a < cat_base) a = cat_base;
@@ -106,6 +128,15 @@ __host__ __device__ inline uint32_t run_chunk_owner(uint32_t nc, uint32_t cq, ui
   while (i > 0 && run_first_chunk(nc, cq, cr, i) > p) --i;
   while (i + 1 < nc && run_first_chunk(nc, cq, cr, i + 1) <= p) ++i;
   return i;
+}
+// The last CTA that works on tile T of an operation with n_groups chunks per tile.
+__host__ __device__ inline uint32_t op_last_cta(uint32_t nc, uint32_t cq, uint32_t cr, uint32_t cat_base, uint32_t n_groups, uint32_t T) {
+  if (cr & kSplitAligned) {
+    uint32_t c0, c1;
+    aligned_tile_ctas(nc, cr & ~kSplitAligned, T, c0, c1);
+    return c1 - 1;
+  }
+  return run_chunk_owner(nc, cq, cr, cat_base + T * n_groups + n_groups - 1);
 }
 // Host: split a run of `run_total` chunks among ncta CTAs.
 inline void run_split(uint32_t run_total, uint32_t ncta, uint32_t& nc, uint32_t& cq, uint32_t& cr) {

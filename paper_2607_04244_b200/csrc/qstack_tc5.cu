@@ -184,17 +184,30 @@ __device__ __forceinline__ void wait_shared_gt(volatile int* p, int seen, const 
 // The fields of a descriptor that every role needs at every operation (two 16-byte loads through
 // the read-only path: the descriptors do not change while the kernel runs).
 struct OpHead {
-  uint32_t nc, cq, cr, cat_base, total_chunks;
+  uint32_t start, end;     // this CTA's chunks of the operation (per matrix); start >= end: none
+  uint32_t last;           // the last CTA that works on the tile of chunk end - 1
+  uint32_t total_chunks;
   int n_groups, n_tiles, flags;
 };
-// (the kernel copies the first 32 bytes of every descriptor into shared memory when it starts)
+// (when it starts, the kernel resolves the split of every operation for its own CTA and keeps the
+// result in shared memory: no role repeats the split's divisions at every operation)
 __device__ __forceinline__ OpHead load_head(const uint4* s_heads, int j) {
   const uint4 a = s_heads[2 * j];
   const uint4 b = s_heads[2 * j + 1];
   OpHead h;
-  h.nc = a.x; h.cq = a.y; h.cr = a.z; h.cat_base = a.w;
+  h.start = a.x; h.end = a.y; h.last = a.z;
   h.total_chunks = b.x; h.n_groups = (int)b.y; h.n_tiles = (int)b.z; h.flags = (int)b.w;
   return h;
+}
+__device__ __forceinline__ void resolve_head(const StackParams& sp, int j, uint32_t cta, uint4* s_heads) {
+  const uint4 a = __ldg(reinterpret_cast<const uint4*>(sp.ops + j));
+  const uint4 b = __ldg(reinterpret_cast<const uint4*>(sp.ops + j) + 1);
+  const uint32_t Gn = b.y;
+  uint32_t lo = 0, hi = 0, last = 0;
+  op_local_range(a.x, a.y, a.z, a.w, b.x, cta, lo, hi);
+  if (lo < hi) last = op_last_cta(a.x, a.y, a.z, a.w, Gn, (hi - 1) / Gn);
+  s_heads[2 * j] = make_uint4(lo, hi, last, 0u);
+  s_heads[2 * j + 1] = b;
 }
 template <typename T>
 __device__ __forceinline__ T* ldg_ptr(T* const* p) {
@@ -399,8 +412,7 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
     tmem_alloc(s_tmem, TMEM_COLS);
     tmem_relinquish();
   }
-  for (int i = tid; i < 2 * sp.n_ops; i += st_threads(RING, PAIRED))
-    s_heads[i] = __ldg(reinterpret_cast<const uint4*>(ops + (i >> 1)) + (i & 1));
+  for (int i = tid; i < sp.n_ops; i += st_threads(RING, PAIRED)) resolve_head(sp, i, cta, s_heads);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -415,7 +427,7 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
       for (int j = 0; j < sp.n_ops; ++j) {
         const OpHead h = load_head(s_heads, j);
         uint32_t start, end;
-        op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
+        start = h.start; end = h.end;
         if (start >= end) continue;
         if (sp.ablate & 1) continue;
         const uint8_t* p0 = ldg_ptr(&ops[j].packed0);
@@ -451,7 +463,7 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
         // operations this CTA has no chunk of need nothing from it: a later operation it takes part in
         // waits for its own predecessor, which cannot be complete before everything ahead of it is
         uint32_t lo, hi;
-        op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, lo, hi);
+        lo = h.start; hi = h.end;
         if (lo >= hi) continue;
       }
       // the unpack warps read the descriptor from shared memory (two slots, alternating); a slot is
@@ -494,7 +506,7 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
       }
       const int prologue = __ldg(&ops[j].prologue);
       uint32_t start, end;
-      op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
+      start = h.start; end = h.end;
       if (prologue != 0 && start < end) {
         // 1/rms of every row from the per-tile sums of squares the producer operation left
         // (fixed order: tiles of one parity ascending, then even + odd)
@@ -530,7 +542,7 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
       for (int j = 0; j < sp.n_ops; ++j) {
         const OpHead h = load_head(s_heads, j);
         uint32_t start, end;
-        op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
+        start = h.start; end = h.end;
         if (start >= end) continue;
         const uint16_t* in0 = ldg_ptr(&ops[j].in0);
         const int ld_in = __ldg(&ops[j].ld_in);
@@ -577,7 +589,7 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
       for (int j = 0; j < sp.n_ops; ++j) {
         const OpHead h = load_head(s_heads, j);
         uint32_t start, end;
-        op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
+        start = h.start; end = h.end;
         if (start >= end) continue;
         const bool dual = (h.flags & kOpDual) != 0;
         const uint32_t Gn = (uint32_t)h.n_groups;
@@ -665,7 +677,7 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
     for (int j = 0; j < sp.n_ops; ++j) {
       const OpHead h = load_head(s_heads, j);
       uint32_t start, end;
-      op_local_range(h.nc, h.cq, h.cr, h.cat_base, h.total_chunks, cta, start, end);
+      start = h.start; end = h.end;
       if (start >= end) continue;
       // the watcher has put the descriptor into shared memory (normally long before)
       if (lane == 0) wait_shared_gt(s_descrdy, j, wc, 13);
@@ -844,7 +856,7 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
         if (!whole && !(sp.ablate & 8)) {
           // ---- owner of a split tile: its own partial stays in registers; the others' are added in
           //      CTA order once their flags for this row are up (lane q polls contributor q) ----
-          const uint32_t last = run_chunk_owner(h.nc, h.cq, h.cr, h.cat_base + T * Gn + Gn - 1);
+          const uint32_t last = h.last;                  // (a split tile that a piece begins is the piece's last tile)
           for (uint32_t i = cta + 1 + lane; i <= last; i += 32) wait_global<false>(&row_flag[16 * i], (int)tag, wc, 10);
           __syncwarp();
           fence_gpu();                                     // acquire: the contributors' rows

@@ -119,6 +119,33 @@ def test_full_size_layers_teacher_forced(ql):
         check_layer(l, bufs, weights, qsynth.LAYER_SHAPES, g, qsynth.Q_DIM)
 
 
+@pytest.mark.parametrize("g", [128, 64])
+def test_full_size_layer_under_every_split(ql, g):
+    """The split of a chained operation decides which thread blocks share a tile and in which
+    order partial rows are added, never what is computed: one full-size layer under the even
+    split, the aligned split without and with the owner's extra chunks, and an extra so large
+    that it is clipped; every linear teacher-forced against the oracle each time."""
+    M = 16
+    ops, bufs, weights, _pk = build_stack(ql, 1, qsynth.LAYER_SHAPES, M, g, qsynth.Q_DIM, layer_ids=[3])
+    ws = ql.new_workspace(M, qsynth.MLP_DIM)
+    arr = ql.make_ops(ops)
+    try:
+        for extra in (-2, 0, 1, 4, 9, 1000):
+            ql.ql_debug_set_owner_extra(extra)
+            kt, kg = qsynth.LAYER_SHAPES["down"][1] // 128, qsynth.LAYER_SHAPES["down"][0] // g
+            assert ql.ql_plan_chain_split(kt, kg, 148, 0)["aligned"] == (extra >= 0)
+            for v in bufs.values():
+                for t in v:
+                    t.fill_(0x7FC0)                      # NaN: nothing of an earlier run can pass for a result
+            bufs["h"][0].copy_(dev_u16(qsynth.stack_h0(M)))
+            ql.qlinear_stack_w4a16(arr, ws)
+            torch.cuda.synchronize()
+            assert ql.ql_device_status(ws) == ql.QL_OK
+            check_layer(0, bufs, weights, qsynth.LAYER_SHAPES, g, qsynth.Q_DIM)
+    finally:
+        ql.ql_debug_set_owner_extra(-1)
+
+
 def test_drafter_layers_symmetric_full_size(ql):
     """The second workload: drafter layers (group-wise symmetric INT4, groups of 128, M = 16; paper
     Sections 3.2 and 3.3) through the same launcher, zero == NULL at the boundary.  Two of the five

@@ -149,6 +149,50 @@ def test_stream_k_split_is_balanced_contiguous_and_invertible(ql):
             assert firsts[o] <= c < firsts[o + 1], (total, ncta, c, o)
 
 
+def test_chain_split_aligned_where_tiles_can_have_thread_blocks_of_their_own(ql):
+    """Chained operations: with at most ncta / 2 tiles and two chunks per thread block the aligned
+    split is taken - pieces tile [0, total), no piece crosses a tile boundary, the thread blocks of
+    a tile are consecutive, the first of them (the owner) has the extra chunks, and `last_cta` is
+    the last thread block of the piece's tile.  Otherwise the even split, as before."""
+    import random
+    rnd = random.Random(11)
+    try:
+        for extra in (-1, 0, 3, 7, 500, -2):
+            ql.ql_debug_set_owner_extra(extra)
+            cases = [(20, 32, 148), (20, 76, 148), (48, 20, 148), (76, 20, 148), (1187, 20, 148), (20, 3, 148), (74, 4, 148),
+                     (74, 3, 148), (1, 40, 148), (1, 400, 148), (3, 1000, 160), (20, 64, 132)]
+            cases += [(rnd.randint(1, 90), rnd.randint(1, 160), rnd.randint(2, 160)) for _ in range(40)]
+            for nt, gn, ncta in cases:
+                rs = [ql.ql_plan_chain_split(nt, gn, ncta, i) for i in range(ncta)]
+                total, pos = nt * gn, 0
+                for r in rs:
+                    if r["lo"] < r["hi"]:
+                        assert r["lo"] == pos
+                        pos = r["hi"]
+                assert pos == total, (nt, gn, ncta, extra)
+                most = -(-ncta // nt)
+                want_aligned = extra >= -1 and 2 * nt <= ncta and gn >= 2 * most
+                assert all(r["aligned"] == want_aligned for r in rs)
+                if not want_aligned:
+                    nc = min(ncta, total)
+                    assert [r["lo"] for r in rs[:nc]] == [(i * total) // nc for i in range(nc)]
+                    continue
+                e = 4 if extra == -1 else extra
+                for T in range(nt):
+                    ctas = [i for i, r in enumerate(rs) if r["lo"] // gn == T]
+                    assert ctas == list(range(ctas[0], ctas[-1] + 1)) and len(ctas) >= 2
+                    assert ctas[0] == (T * ncta) // nt and ctas[-1] + 1 == ((T + 1) * ncta) // nt
+                    sizes = [rs[i]["hi"] - rs[i]["lo"] for i in ctas]
+                    assert all((rs[i]["hi"] - 1) // gn == T and rs[i]["last_cta"] == ctas[-1] for i in ctas)
+                    assert min(sizes) >= 1 and sum(sizes) == gn
+                    e_eff = min(e, gn - most)
+                    rest = sizes[1:]
+                    assert max(rest) - min(rest) <= 1
+                    assert sizes[0] == e_eff + (gn - e_eff) // len(ctas)
+    finally:
+        ql.ql_debug_set_owner_extra(-1)
+
+
 def test_verification_tail_argument_errors(ql):
     P = 0x100000
     base = dict(kind=ql.QL_OP_LINEAR, M=16, K=512, N=256, g=128, ld_in=512, ld_out=256, packed=P, in0=P, out=P)
