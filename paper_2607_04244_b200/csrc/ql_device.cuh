@@ -216,6 +216,29 @@ __device__ __forceinline__ uint32_t codes_minus_zero(uint32_t masked, uint32_t z
   return *reinterpret_cast<uint32_t*>(&r);
 }
 
+// One 32-bit word of the packed layout (8 codes: extraction s takes the nibbles at bits 4s and
+// 16 + 4s) -> four bf16x2 registers of the exact integers code - z.  Written in PTX so that the
+// instruction sequence is the intended one (3 shifts, 4 and-or LOP3s, 4 packed subtractions); the
+// compiler's own selection for the C++ form was 15 % slower in the mma.sync kernel's chunk loop.
+__device__ __forceinline__ void unpack_word(uint32_t w, uint32_t zbias, uint32_t& b0, uint32_t& b1, uint32_t& b2, uint32_t& b3) {
+  asm("{\n\t"
+      ".reg .b32 w1, w2, w3;\n\t"
+      "shr.u32 w1, %4, 4;\n\t"
+      "shr.u32 w2, %4, 8;\n\t"
+      "shr.u32 w3, %4, 12;\n\t"
+      "lop3.b32 %0, %4, 0x000f000f, 0x43004300, 0xea;\n\t"
+      "lop3.b32 %1, w1, 0x000f000f, 0x43004300, 0xea;\n\t"
+      "lop3.b32 %2, w2, 0x000f000f, 0x43004300, 0xea;\n\t"
+      "lop3.b32 %3, w3, 0x000f000f, 0x43004300, 0xea;\n\t"
+      "sub.bf16x2 %0, %0, %5;\n\t"
+      "sub.bf16x2 %1, %1, %5;\n\t"
+      "sub.bf16x2 %2, %2, %5;\n\t"
+      "sub.bf16x2 %3, %3, %5;\n\t"
+      "}"
+      : "=&r"(b0), "=&r"(b1), "=&r"(b2), "=&r"(b3)
+      : "r"(w), "r"(zbias));
+}
+
 // ---- tcgen05 (5th-generation tensor core, tensor memory) ----------------------------------------
 // Tensor-memory addresses are (lane << 16) | column.  A warp may touch only lanes
 // [32*(warp%4), 32*(warp%4)+32).
@@ -283,9 +306,7 @@ __host__ __device__ constexpr uint32_t tc_idesc_bf16_m128(uint32_t n) {
 __device__ __forceinline__ void unpack_codes32(const uint4 w4, uint32_t zbias, uint32_t (&v)[16]) {
   const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
-  for (int j = 0; j < 4; ++j)
-#pragma unroll
-    for (int s = 0; s < 4; ++s) v[4 * j + s] = codes_minus_zero((ww[j] >> (4 * s)) & 0x000f000fu, zbias);
+  for (int j = 0; j < 4; ++j) unpack_word(ww[j], zbias, v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
 }
 
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t pair) { return __uint_as_float(pair << 16); }

@@ -74,10 +74,8 @@ __device__ __forceinline__ void compute_chunk(const uint8_t* __restrict__ st, co
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const uint32_t w = W[(c * 128 + n0 + 8 * j + g8) * 4 + t];
-      const uint32_t b0 = codes_minus_zero(w & 0x000f000fu, zb[j]);
-      const uint32_t b1 = codes_minus_zero((w >> 4) & 0x000f000fu, zb[j]);
-      const uint32_t b2 = codes_minus_zero((w >> 8) & 0x000f000fu, zb[j]);
-      const uint32_t b3 = codes_minus_zero((w >> 12) & 0x000f000fu, zb[j]);
+      uint32_t b0, b1, b2, b3;
+      unpack_word(w, zb[j], b0, b1, b2, b3);
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) {
         mma_bf16_16816(P[j][mt], xa[mt].x, xb[mt].x, xa[mt].y, xb[mt].y, b0, b1);
@@ -204,6 +202,27 @@ __global__ void __launch_bounds__(mma_kgroups(MT) * 128 + 32, 1) qlinear_mma_ker
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[j][mt][e] = 0.f;
 
+    if (MT <= 2 && XP == 0) {
+      // resident X (kernels for up to 32 rows): the k-group walks its own chunks (every KG-th) with ring stage, phase and X slot
+      // carried along - no division and no skipped iteration per chunk
+      uint32_t ci = ((uint32_t)kg + KG - (it % KG)) % KG;
+      const uint32_t itk = it + ci;
+      uint32_t s = itk % NS, ph = (itk / NS) & 1;
+      uint32_t xk = (g0 + ci + Gn - g_first) % Gn;
+      const uint8_t* stp = ring + (size_t)s * stage;
+      const uint8_t* xp = xbuf + (size_t)xk * xslot;
+      for (; ci < nch; ci += KG) {
+        mbar_wait(&full[s], ph, s_abort, p.ws.status);
+        if (!(p.ablate & 1)) compute_chunk<MT, G>(stp, xp, wn, g8, t, acc);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[s]);
+        s += KG; stp += (size_t)KG * stage;
+        while (s >= (uint32_t)NS) { s -= NS; ph ^= 1; stp -= (size_t)NS * stage; }
+        xk += KG; xp += (size_t)KG * xslot;
+        while (xk >= Gn) { xk -= Gn; xp -= (size_t)Gn * xslot; }
+      }
+      it += nch;
+    } else
     for (uint32_t ci = 0; ci < nch; ++ci, ++it) {
       if (XP != 0 && it % XP == 0) {
         named_bar_sync(1, NCONS);                          // every consumer is done with the previous phase's X
