@@ -29,7 +29,7 @@ static std::atomic<uint64_t> g_wait_ns{kWaitBudgetNs};    // budget of the stack
 // debug hook changes: a remembered plan is valid only while nothing of that happened since it was staged.
 static std::atomic<uint64_t> g_desc_gen{1};
 static std::atomic<int> g_no_release_op{-1};              // test hook: fused operation that does not publish its tiles
-constexpr int kOwnerExtraChunks = 4;                      // aligned split: chunks the owner of a tile takes beyond an even share
+constexpr int kOwnerExtraChunks = 1;                      // aligned split: chunks the owner of a tile takes beyond an even share
 static std::atomic<int> g_owner_extra{kOwnerExtraChunks}; // (measurement hook ql_debug_set_owner_extra; negative: even split everywhere)
 static std::atomic<int> g_ablate{0};                      // timing experiments: phases of the stack kernel switched off
 static std::atomic<uint64_t*> g_timeline{nullptr};        // device buffer for the in-kernel timeline (QL_TIMELINE builds)
@@ -223,7 +223,8 @@ static void split_one_stream(std::vector<MegaOp>& mega, int ncta) {
 // chunks for each of them (the fused qkv, attention-output and MLP-down projections of a verify
 // step: 48 or 20 tiles on 148 CTAs), the aligned split is taken: no CTA meets two tiles, and the
 // first CTA of a tile - its owner, which has to wait for the others' partial rows before it can
-// finish the tile - unpacks g_owner_extra chunks more than they do in the meantime.  Otherwise
+// finish the tile - unpacks g_owner_extra chunks more than they do in the meantime (one chunk:
+// the rows travel as {value, tag} pairs and are there a microsecond after the contributor's last MMA).  Otherwise
 // (gate/up pairs: 76 double tiles; the LM head) the chunks are shared out evenly and pieces cross
 // tile boundaries.
 static void chain_split(MegaOp& m, int ncta) {

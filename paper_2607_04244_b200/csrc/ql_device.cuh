@@ -23,6 +23,7 @@ __host__ __device__ constexpr uint32_t align128(uint32_t x) { return (x + 127u) 
 //                                                                [kMaxOps][16][32]
 // -- everything above is zero between calls (ql_workspace_init zeroes it once, kernels restore it) --
 // then            operation descriptors of the stack kernel      [kMaxOps * kOpDescBytes]
+// then            partial tiles of the stack kernel as {value, tag} pairs   [kWsPairBytes]
 // then            row sums of squares per tile, two buffers      [2][tiles][16] fp32
 // then            fp32 product silu(gate)*up of a dual operation, dense [16][N]   [16][tiles*128]
 // then            arg-max candidates                             [tiles][m_pad] (value, index)
@@ -37,6 +38,10 @@ constexpr int kOpDescBytes = 160;
 constexpr int kWsHeaderBytes = 256;
 constexpr size_t kWsControlBytes = kWsHeaderBytes + (size_t)kFlagWords * 4 + (size_t)kMaxOps * 16 * kOpDoneStride * 4;
 constexpr size_t kWsDescBytes = (size_t)kMaxOps * kOpDescBytes;
+// Partial tiles of the stack kernel: {value, tag} pairs of 8 bytes, [2 sets][160 CTAs][2 matrices][16 rows][128].
+// The region is written by that kernel only and sits at a fixed offset, so that a word in it is
+// either zero (ql_workspace_init) or carries the tag of the launch and operation that wrote it.
+constexpr size_t kWsPairBytes = (size_t)kMaxCtas * 2 * 16 * 128 * 8;
 
 struct Workspace {
   int* status;
@@ -49,6 +54,7 @@ struct Workspace {
   float* act;        // [16][N] of the dual operation that wrote it, dense (capacity 16 * n_tiles * 128)
   float2* cand;      // .x = value, .y = index bits
   float* slots;
+  uint64_t* pairs;   // partial tiles of the stack kernel, {value, tag} pairs
   int n_tiles;       // tile capacity the regions were carved for
 };
 
@@ -59,7 +65,7 @@ __host__ __device__ inline size_t ws_cand_bytes(int n_tiles, int m_pad) { return
 __host__ __device__ inline size_t ws_slot_floats(int m_pad) { return (size_t)2 * m_pad * kTileN; }   // two matrices
 __host__ __device__ inline size_t ws_act_bytes(int n_tiles) { return (size_t)16 * n_tiles * kTileN * 4; }
 __host__ __device__ inline size_t ws_total_bytes(int n_tiles, int m_pad) {
-  return kWsControlBytes + kWsDescBytes + ws_ssq_bytes(n_tiles) + ws_act_bytes(n_tiles) + ws_cand_bytes(n_tiles, m_pad) +
+  return kWsControlBytes + kWsDescBytes + kWsPairBytes + ws_ssq_bytes(n_tiles) + ws_act_bytes(n_tiles) + ws_cand_bytes(n_tiles, m_pad) +
          (size_t)kMaxCtas * 2 * ws_slot_floats(m_pad) * 4;
 }
 // Carves the regions for a tile capacity and row padding.  Within one workspace every call must
@@ -74,7 +80,8 @@ __host__ __device__ inline Workspace ws_carve(void* base, int n_tiles, int m_pad
   w.tile_cnt = (int*)(p + kWsHeaderBytes);
   w.op_done = w.tile_cnt + kFlagWords;
   w.desc = (uint8_t*)(p + kWsControlBytes);
-  p += kWsControlBytes + kWsDescBytes;
+  w.pairs = (uint64_t*)(p + kWsControlBytes + kWsDescBytes);
+  p += kWsControlBytes + kWsDescBytes + kWsPairBytes;
   w.ssq = (float*)p;
   p += ws_ssq_bytes(n_tiles);
   w.act = (float*)p;

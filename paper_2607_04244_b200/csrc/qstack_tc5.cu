@@ -82,6 +82,17 @@ __device__ __forceinline__ void red_relaxed_add(int* p, int v) {
   asm volatile("red.relaxed.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void fence_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
+// Partial rows travel between CTAs as {value, tag} pairs of 8 bytes: a 64-bit access is single-copy
+// atomic, so a pair whose tag is the expected one carries its value - no fence after the stores,
+// no flag, no fence before the loads.  Two pairs per 16-byte access.
+__device__ __forceinline__ void st_pairs(uint64_t* p, float a, float b, uint32_t tag) {
+  const uint64_t u0 = ((uint64_t)tag << 32) | (uint64_t)__float_as_uint(a);
+  const uint64_t u1 = ((uint64_t)tag << 32) | (uint64_t)__float_as_uint(b);
+  asm volatile("st.relaxed.gpu.global.v2.b64 [%0], {%1, %2};" ::"l"(p), "l"(u0), "l"(u1) : "memory");
+}
+__device__ __forceinline__ void ld_pairs(const uint64_t* p, uint64_t& u0, uint64_t& u1) {
+  asm volatile("ld.relaxed.gpu.global.v2.b64 {%0, %1}, [%2];" : "=l"(u0), "=l"(u1) : "l"(p) : "memory");
+}
 
 // In-kernel timeline (builds with -DQL_TIMELINE): thread 0 of a CTA stamps the phases of every
 // operation, the watcher's lane 0 the moment it saw the previous operation complete.
@@ -832,51 +843,68 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
         if ((sp.ablate & 8) && !whole && !finish) { pos += nch; continue; }
         pos += nch;
         const int nmat = dual ? 2 : 1;
-        int* row_flag = sp.ws.tile_cnt + kMaxTiles + (j & 1) * (16 * kSetCtas) + rw;   // flag of (CTA i, row r) at [16 i + r] of the set j & 1, behind the tile counters of the single-launch kernels
-        float* set_slots = sp.ws.slots + (size_t)(j & 1) * kSetCtas * kSlotWords;
-        float* my_slot = set_slots + (size_t)cta * kSlotWords;
+        // partial rows of split tiles: pairs [set j & 1][CTA][matrix][row][column]
+        uint64_t* set_pairs = sp.ws.pairs + (size_t)(j & 1) * kSetCtas * kSlotWords;
+        const size_t row_off = (size_t)rw * kTileN + 4 * lane;
 
         if (!whole && !finish) {
-          // ---- contributor: row r of its partial tile, one fence over the warp's stores, then the
-          //      row's flag.  (A run that does not begin its tile meets it in its first segment, so
-          //      one slot per CTA is enough.) ----
+          // ---- contributor: row r of its partial tile as {value, tag} pairs; nothing else to do.
+          //      (A run that does not begin its tile meets it in its first segment, so one slot
+          //      per CTA is enough.) ----
           for (int mt = 0; mt < nmat; ++mt) {
             const float* f = mt ? f1 : f0;
-            __stcg(reinterpret_cast<float4*>(my_slot + (size_t)(mt * MP + rw) * kTileN + 4 * lane), make_float4(f[0], f[1], f[2], f[3]));
-          }
-          __syncwarp();
-          if (lane == 0) {
-            fence_gpu();
-            st_relaxed(&row_flag[16 * cta], (int)tag);
+            uint64_t* dst = set_pairs + (size_t)cta * kSlotWords + (size_t)mt * MP * kTileN + row_off;
+            st_pairs(dst, f[0], f[1], tag);
+            st_pairs(dst + 2, f[2], f[3], tag);
           }
           if (pos - nch == start) QL_STAMP(6);
           if (pos == end) QL_STAMP(14);
           continue;
         }
         if (!whole && !(sp.ablate & 8)) {
-          // ---- owner of a split tile: its own partial stays in registers; the others' are added in
-          //      CTA order once their flags for this row are up (lane q polls contributor q) ----
+          // ---- owner of a split tile: its own partial stays in registers; the others' rows are
+          //      polled until every pair carries this operation's tag, four contributors at a
+          //      time, and added in CTA order ----
           const uint32_t last = h.last;                  // (a split tile that a piece begins is the piece's last tile)
-          for (uint32_t i = cta + 1 + lane; i <= last; i += 32) wait_global<false>(&row_flag[16 * i], (int)tag, wc, 10);
-          __syncwarp();
-          fence_gpu();                                     // acquire: the contributors' rows
           if (pos == end) QL_STAMP(10);
           for (int mt = 0; mt < nmat; ++mt) {
             float* f = mt ? f1 : f0;
-            for (uint32_t i0 = cta + 1; i0 <= last; i0 += 8) {
-              float4 v[8];
+            for (uint32_t i0 = cta + 1; i0 <= last; i0 += 4) {
+              uint64_t u[4][4];
+              uint64_t t0 = 0;
+              uint32_t spins = 0;
+              for (;;) {
 #pragma unroll
-              for (int q = 0; q < 8; ++q) {
-                const uint32_t i = min(i0 + q, last);
-                v[q] = __ldcg(reinterpret_cast<const float4*>(set_slots + (size_t)i * kSlotWords + (size_t)(mt * MP + rw) * kTileN + 4 * lane));
+                for (int q = 0; q < 4; ++q) {
+                  const uint32_t i = min(i0 + q, last);
+                  const uint64_t* src = set_pairs + (size_t)i * kSlotWords + (size_t)mt * MP * kTileN + row_off;
+                  ld_pairs(src, u[q][0], u[q][1]);
+                  ld_pairs(src + 2, u[q][2], u[q][3]);
+                }
+                bool ok = true;
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) ok = ok && ((uint32_t)(u[q][e] >> 32) == tag);
+                if (ok) break;
+                if (spins == 0) {
+                  if (*wc.s_abort) break;
+                  t0 = globaltimer_ns();
+                }
+                if ((++spins & 15u) == 0) {
+                  if (*wc.s_abort) break;
+                  if (globaltimer_ns() - t0 > wc.budget) { wait_fail(wc, 10); break; }
+                }
               }
 #pragma unroll
-              for (int q = 0; q < 8; ++q) {
+              for (int q = 0; q < 4; ++q) {
                 if (i0 + q > last) continue;
-                f[0] += v[q].x; f[1] += v[q].y; f[2] += v[q].z; f[3] += v[q].w;
+                f[0] += __uint_as_float((uint32_t)u[q][0]); f[1] += __uint_as_float((uint32_t)u[q][1]);
+                f[2] += __uint_as_float((uint32_t)u[q][2]); f[3] += __uint_as_float((uint32_t)u[q][3]);
               }
             }
           }
+          __syncwarp();
         }
 
         if (pos == end) QL_STAMP(11);
