@@ -75,6 +75,11 @@ __device__ __forceinline__ int ld_relaxed(const int* p) {
   asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ void st_relaxed(int* p, int v) {
   asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
@@ -507,8 +512,10 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
           const int need = __ldg(&ops[dep].n_tiles);
           wait_global<true>(&sp.ws.op_done[((size_t)dep * 16 + lane) * kOpDoneStride], need, wc, 7);
         }
+        // acquire: everything the finishers published.  One acquire load of the complete counter per
+        // polling lane instead of a fence after the relaxed polls (the fence cost 0.9 us per operation)
+        if (lane < 16 && !(sp.ablate & 256)) ld_acquire(&sp.ws.op_done[((size_t)dep * 16 + lane) * kOpDoneStride]);
         __syncwarp();
-        if (!(sp.ablate & 256)) fence_gpu();             // acquire: everything the finishers published
       }
       QL_STAMP_W(7);
       if (lane == 0) {
