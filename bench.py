@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from an ncu capture of a 3-layer launch of the stack kernel:
 # dram read + write = 160.95 MB for 162.32 MB of algorithmic bytes.  Traffic grows in proportion to the
 # layers streamed (every packed byte crosses HBM once), so a full launch is scaled by this ratio.
-NCU_TRAFFIC_RATIO = 160.95 / 162.32
+NCU_TRAFFIC_RATIO = 161.42 / 162.32
 
 
 # ------------------------------------------------------------------------------------------------

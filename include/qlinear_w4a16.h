@@ -352,7 +352,7 @@ void ql_debug_no_release(int fused_op);
  * buffer: first [160 thread blocks][n_ops][16] SM cycle stamps of thread 0 (0 operation entered,
  * 1 first chunk unpacked, 2 predecessor known complete, 3 X operand built, 4-6 first tile segment
  * drained / exchanged / published, 7 the watcher saw the predecessor complete, 8-14 the same
- * steps of the last tile segment incl. 10 contributors' flags seen, 11 partials added, 12 stores
+ * steps of the last tile segment incl. 10 polling of the contributors' rows starts, 11 partials added, 12 stores
  * issued, 14 published, 15 the publish time in globaltimer ns), then [160][4][8] cycle sums of the
  * unpack groups, [160][4][8] of the MMA issuers, and [160][n_ops] globaltimer ns at which the
  * watcher saw the predecessor complete.  paper_2607_04244_b200/timeline.py sizes and reads it.

@@ -147,9 +147,9 @@ def main():
             "last segment: chunks drained after X built (mean)": mean(e[:, 8] - e[:, 3]),
             "last segment: chunks drained after X built (max)": vmax(e[:, 8] - e[:, 3]),
             "last segment: accumulator exchange (mean)": mean(e[:, 9] - e[:, 8]),
-            "owners of split tiles: wait for the contributors' flags (mean)": mean(e[:, 10] - e[:, 9]),
-            "owners of split tiles: wait for flags (max)": vmax(e[:, 10] - e[:, 9]),
-            "owners: load and add partials (mean)": mean(e[:, 11] - e[:, 10]),
+            "owners of split tiles: exchange -> polling starts (mean)": mean(e[:, 10] - e[:, 9]),
+            "owners of split tiles: exchange -> polling starts (max)": vmax(e[:, 10] - e[:, 9]),
+            "owners: poll and add the contributors' tagged rows (mean)": mean(e[:, 11] - e[:, 10]),
             "finishers: epilogue until stores issued (mean)": mean(e[:, 12] - e[:, 11]),
             "finishers: fence + publish (mean)": mean(e[:, 14] - e[:, 12]),
             "contributors: exchange -> partial sent (mean)": mean(np.where(np.isnan(e[:, 11]), e[:, 14] - e[:, 9], np.nan)),
