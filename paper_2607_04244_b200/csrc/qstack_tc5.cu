@@ -870,45 +870,49 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
         }
         if (!whole && !(sp.ablate & 8)) {
           // ---- owner of a split tile: its own partial stays in registers; the others' rows are
-          //      polled until every pair carries this operation's tag, four contributors at a
-          //      time, and added in CTA order ----
+          //      polled until every pair carries this operation's tag and added in CTA order ----
           const uint32_t last = h.last;                  // (a split tile that a piece begins is the piece's last tile)
           if (pos == end) QL_STAMP(10);
-          for (int mt = 0; mt < nmat; ++mt) {
-            float* f = mt ? f1 : f0;
-            for (uint32_t i0 = cta + 1; i0 <= last; i0 += 4) {
-              uint64_t u[4][4];
-              uint64_t t0 = 0;
-              uint32_t spins = 0;
-              for (;;) {
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                  const uint32_t i = min(i0 + q, last);
-                  const uint64_t* src = set_pairs + (size_t)i * kSlotWords + (size_t)mt * MP * kTileN + row_off;
-                  ld_pairs(src, u[q][0], u[q][1]);
-                  ld_pairs(src + 2, u[q][2], u[q][3]);
-                }
-                bool ok = true;
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-#pragma unroll
-                  for (int e = 0; e < 4; ++e) ok = ok && ((uint32_t)(u[q][e] >> 32) == tag);
-                if (ok) break;
-                if (spins == 0) {
-                  if (*wc.s_abort) break;
-                  t0 = globaltimer_ns();
-                }
-                if ((++spins & 15u) == 0) {
-                  if (*wc.s_abort) break;
-                  if (globaltimer_ns() - t0 > wc.budget) { wait_fail(wc, 10); break; }
-                }
-              }
+          // items = (contributor, matrix) in CTA order, the two matrices of a dual operation side by
+          // side: four items are in flight together (one round of loads covers two contributors of a
+          // gate/up pair or four of a plain linear)
+          const uint32_t items = (last - cta) * (uint32_t)nmat;
+          for (uint32_t k0 = 0; k0 < items; k0 += 4) {
+            uint64_t u[4][4];
+            uint64_t t0 = 0;
+            uint32_t spins = 0;
+            for (;;) {
 #pragma unroll
               for (int q = 0; q < 4; ++q) {
-                if (i0 + q > last) continue;
-                f[0] += __uint_as_float((uint32_t)u[q][0]); f[1] += __uint_as_float((uint32_t)u[q][1]);
-                f[2] += __uint_as_float((uint32_t)u[q][2]); f[3] += __uint_as_float((uint32_t)u[q][3]);
+                const uint32_t k = min(k0 + q, items - 1);
+                const uint32_t i = cta + 1 + (dual ? (k >> 1) : k);
+                const uint32_t mt = dual ? (k & 1u) : 0u;
+                const uint64_t* src = set_pairs + (size_t)i * kSlotWords + (size_t)mt * MP * kTileN + row_off;
+                ld_pairs(src, u[q][0], u[q][1]);
+                ld_pairs(src + 2, u[q][2], u[q][3]);
               }
+              bool ok = true;
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) ok = ok && ((uint32_t)(u[q][e] >> 32) == tag);
+              if (ok) break;
+              if (spins == 0) {
+                if (*wc.s_abort) break;
+                t0 = globaltimer_ns();
+              }
+              if ((++spins & 15u) == 0) {
+                if (*wc.s_abort) break;
+                if (globaltimer_ns() - t0 > wc.budget) { wait_fail(wc, 10); break; }
+              }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              if (k0 + q >= items) continue;
+              const float a0 = __uint_as_float((uint32_t)u[q][0]), a1 = __uint_as_float((uint32_t)u[q][1]);
+              const float a2 = __uint_as_float((uint32_t)u[q][2]), a3 = __uint_as_float((uint32_t)u[q][3]);
+              if (dual && (q & 1)) { f1[0] += a0; f1[1] += a1; f1[2] += a2; f1[3] += a3; }   // (k0 is a multiple of 4: item parity = q parity)
+              else { f0[0] += a0; f0[1] += a1; f0[2] += a2; f0[3] += a3; }
             }
           }
           __syncwarp();
