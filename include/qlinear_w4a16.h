@@ -329,11 +329,11 @@ uint32_t ql_plan_chunk_owner(uint32_t total_chunks, uint32_t ncta, uint32_t chun
  * resolves, for tests).  range[0..1] = the chunks [lo, hi) of thread block `cta` (chunk
  * T * n_groups + G is group G of tile T); range[2] = 1 for the aligned split (at most ncta / 2 tiles
  * and at least two chunks per thread block: every tile has thread blocks of its own, and the first
- * of them, which adds the others' partial rows and finishes the tile, has `owner extra` chunks more
- * than an even share of the rest), 0 for the even stream-K split; range[3] = the last thread block
+ * of them, which adds the others' partial rows and finishes the tile, can be given `owner extra` chunks
+ * more than an even share of the rest), 0 for the even stream-K split; range[3] = the last thread block
  * that works on the tile of chunk hi - 1.  Returns QL_OK, QL_ERR_NULL or QL_ERR_SHAPE.
  * ql_debug_set_owner_extra(e): measurement hook, process-wide, for the calls that follow: the
- * owner's extra chunks (-1: the default of 1; below -1: even split everywhere). */
+ * owner's extra chunks (-1: the default of 0; below -1: even split everywhere). */
 int ql_plan_chain_split(int n_tiles, int n_groups, int ncta, int cta, uint32_t range[4]);
 void ql_debug_set_owner_extra(int chunks);
 

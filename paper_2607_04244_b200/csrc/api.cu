@@ -29,7 +29,7 @@ static std::atomic<uint64_t> g_wait_ns{kWaitBudgetNs};    // budget of the stack
 // debug hook changes: a remembered plan is valid only while nothing of that happened since it was staged.
 static std::atomic<uint64_t> g_desc_gen{1};
 static std::atomic<int> g_no_release_op{-1};              // test hook: fused operation that does not publish its tiles
-constexpr int kOwnerExtraChunks = 1;                      // aligned split: chunks the owner of a tile takes beyond an even share
+constexpr int kOwnerExtraChunks = 0;                      // aligned split: chunks the owner of a tile takes beyond an even share
 static std::atomic<int> g_owner_extra{kOwnerExtraChunks}; // (measurement hook ql_debug_set_owner_extra; negative: even split everywhere)
 static std::atomic<int> g_ablate{0};                      // timing experiments: phases of the stack kernel switched off
 static std::atomic<uint64_t*> g_timeline{nullptr};        // device buffer for the in-kernel timeline (QL_TIMELINE builds)
@@ -221,12 +221,12 @@ static void split_one_stream(std::vector<MegaOp>& mega, int ncta) {
 
 // Split of a chained operation.  Where every tile can have at least two CTAs of its own and two
 // chunks for each of them (the fused qkv, attention-output and MLP-down projections of a verify
-// step: 48 or 20 tiles on 148 CTAs), the aligned split is taken: no CTA meets two tiles, and the
-// first CTA of a tile - its owner, which has to wait for the others' partial rows before it can
-// finish the tile - unpacks g_owner_extra chunks more than they do in the meantime (one chunk:
-// the rows travel as {value, tag} pairs and are there a microsecond after the contributor's last MMA).  Otherwise
-// (gate/up pairs: 76 double tiles; the LM head) the chunks are shared out evenly and pieces cross
-// tile boundaries.
+// step: 48 or 20 tiles on 148 CTAs), the aligned split is taken: no CTA meets two tiles.  The
+// first CTA of a tile - its owner, which adds the others' partial rows and finishes the tile - can
+// be given g_owner_extra chunks more than an even share of the rest; that paid while the rows
+// travelled behind a fence and a flag (4 chunks) and no longer does (0: the rows signal themselves
+// and arrive while the owner passes its own tile end).  Otherwise (gate/up pairs: 76 double tiles;
+// the LM head) the chunks are shared out evenly and pieces cross tile boundaries.
 static void chain_split(MegaOp& m, int ncta) {
   m.cat_base = 0;
   const uint32_t nt = (uint32_t)m.n_tiles, Gn = (uint32_t)m.n_groups, nc = (uint32_t)ncta;
@@ -536,8 +536,12 @@ int ql_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
   if (workspace_bytes < kWsControlBytes) return QL_ERR_WORKSPACE;
   if (!aligned16(workspace)) return QL_ERR_ALIGN;
   g_desc_gen.fetch_add(1, std::memory_order_relaxed);     // staged descriptors are gone
-  // everything, not only the control words: the partial-tile slots carry tags, and a stale tag must never look valid
+  // everything, not only the control words; the stack kernel's partial-tile region holds "nothing waiting" (all ones)
   if (cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) return QL_ERR_CUDA;
+  const size_t parts_at = kWsControlBytes + kWsDescBytes;
+  if (workspace_bytes >= parts_at + kWsPairBytes &&
+      cudaMemsetAsync(static_cast<char*>(workspace) + parts_at, 0xFF, kWsPairBytes, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return QL_ERR_CUDA;
   return QL_OK;
 }
 

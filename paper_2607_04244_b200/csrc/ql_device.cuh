@@ -23,7 +23,7 @@ __host__ __device__ constexpr uint32_t align128(uint32_t x) { return (x + 127u) 
 //                                                                [kMaxOps][16][32]
 // -- everything above is zero between calls (ql_workspace_init zeroes it once, kernels restore it) --
 // then            operation descriptors of the stack kernel      [kMaxOps * kOpDescBytes]
-// then            partial tiles of the stack kernel as {value, tag} pairs   [kWsPairBytes]
+// then            partial tiles of the stack kernel (self-signalling values)   [kWsPairBytes]
 // then            row sums of squares per tile, two buffers      [2][tiles][16] fp32
 // then            fp32 product silu(gate)*up of a dual operation, dense [16][N]   [16][tiles*128]
 // then            arg-max candidates                             [tiles][m_pad] (value, index)
@@ -38,10 +38,12 @@ constexpr int kOpDescBytes = 160;
 constexpr int kWsHeaderBytes = 256;
 constexpr size_t kWsControlBytes = kWsHeaderBytes + (size_t)kFlagWords * 4 + (size_t)kMaxOps * 16 * kOpDoneStride * 4;
 constexpr size_t kWsDescBytes = (size_t)kMaxOps * kOpDescBytes;
-// Partial tiles of the stack kernel: {value, tag} pairs of 8 bytes, [2 sets][160 CTAs][2 matrices][16 rows][128].
-// The region is written by that kernel only and sits at a fixed offset, so that a word in it is
-// either zero (ql_workspace_init) or carries the tag of the launch and operation that wrote it.
-constexpr size_t kWsPairBytes = (size_t)kMaxCtas * 2 * 16 * 128 * 8;
+// Partial tiles of the stack kernel, fp32 [2 sets][160 CTAs][2 matrices][16 rows][128].  A word is either
+// kPartEmpty (ql_workspace_init fills the region with it, and the CTA that has added a partial row puts
+// it back) or a value a contributor stored: the value is its own signal, no flag and no fence travel
+// with it.  The region is written by that kernel only and sits at a fixed offset.
+constexpr uint32_t kPartEmpty = 0xFFFFFFFFu;         // a NaN no arithmetic produces (stores replace it by the canonical NaN)
+constexpr size_t kWsPairBytes = (size_t)kMaxCtas * 2 * 16 * 128 * 4;
 
 struct Workspace {
   int* status;
@@ -54,7 +56,7 @@ struct Workspace {
   float* act;        // [16][N] of the dual operation that wrote it, dense (capacity 16 * n_tiles * 128)
   float2* cand;      // .x = value, .y = index bits
   float* slots;
-  uint64_t* pairs;   // partial tiles of the stack kernel, {value, tag} pairs
+  float* parts;      // partial tiles of the stack kernel (kPartEmpty where nothing is waiting)
   int n_tiles;       // tile capacity the regions were carved for
 };
 
@@ -80,7 +82,7 @@ __host__ __device__ inline Workspace ws_carve(void* base, int n_tiles, int m_pad
   w.tile_cnt = (int*)(p + kWsHeaderBytes);
   w.op_done = w.tile_cnt + kFlagWords;
   w.desc = (uint8_t*)(p + kWsControlBytes);
-  w.pairs = (uint64_t*)(p + kWsControlBytes + kWsDescBytes);
+  w.parts = (float*)(p + kWsControlBytes + kWsDescBytes);
   p += kWsControlBytes + kWsDescBytes + kWsPairBytes;
   w.ssq = (float*)p;
   p += ws_ssq_bytes(n_tiles);

@@ -87,16 +87,22 @@ __device__ __forceinline__ void red_relaxed_add(int* p, int v) {
   asm volatile("red.relaxed.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void fence_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
-// Partial rows travel between CTAs as {value, tag} pairs of 8 bytes: a 64-bit access is single-copy
-// atomic, so a pair whose tag is the expected one carries its value - no fence after the stores,
-// no flag, no fence before the loads.  Two pairs per 16-byte access.
-__device__ __forceinline__ void st_pairs(uint64_t* p, float a, float b, uint32_t tag) {
-  const uint64_t u0 = ((uint64_t)tag << 32) | (uint64_t)__float_as_uint(a);
-  const uint64_t u1 = ((uint64_t)tag << 32) | (uint64_t)__float_as_uint(b);
-  asm volatile("st.relaxed.gpu.global.v2.b64 [%0], {%1, %2};" ::"l"(p), "l"(u0), "l"(u1) : "memory");
+// Partial rows travel between CTAs as plain fp32 words that signal themselves: a word of the slot is
+// kPartEmpty until the contributor's value lands (32-bit accesses are single-copy atomic), and the
+// owner puts kPartEmpty back once it has added the row - no fence after the stores, no flag, no fence
+// before the loads.  The put-back is ordered before the slot's next use (two operations later, or
+// the next launch) by the owner's own publish fence and the chain of waits behind it.
+__device__ __forceinline__ void st_part(float* p, float a, float b, float c, float d) {
+  uint32_t u0 = __float_as_uint(a), u1 = __float_as_uint(b), u2 = __float_as_uint(c), u3 = __float_as_uint(d);
+  u0 = u0 == kPartEmpty ? 0x7FFFFFFFu : u0; u1 = u1 == kPartEmpty ? 0x7FFFFFFFu : u1;   // (a NaN stays a NaN)
+  u2 = u2 == kPartEmpty ? 0x7FFFFFFFu : u2; u3 = u3 == kPartEmpty ? 0x7FFFFFFFu : u3;
+  asm volatile("st.relaxed.gpu.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(u0), "r"(u1), "r"(u2), "r"(u3) : "memory");
 }
-__device__ __forceinline__ void ld_pairs(const uint64_t* p, uint64_t& u0, uint64_t& u1) {
-  asm volatile("ld.relaxed.gpu.global.v2.b64 {%0, %1}, [%2];" : "=l"(u0), "=l"(u1) : "l"(p) : "memory");
+__device__ __forceinline__ void ld_part(const float* p, uint32_t (&u)[4]) {
+  asm volatile("ld.relaxed.gpu.global.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]) : "l"(p) : "memory");
+}
+__device__ __forceinline__ void clear_part(float* p) {
+  asm volatile("st.relaxed.gpu.global.v4.b32 [%0], {%1, %1, %1, %1};" ::"l"(p), "r"(kPartEmpty) : "memory");
 }
 
 // In-kernel timeline (builds with -DQL_TIMELINE): thread 0 of a CTA stamps the phases of every
@@ -850,19 +856,16 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
         if ((sp.ablate & 8) && !whole && !finish) { pos += nch; continue; }
         pos += nch;
         const int nmat = dual ? 2 : 1;
-        // partial rows of split tiles: pairs [set j & 1][CTA][matrix][row][column]
-        uint64_t* set_pairs = sp.ws.pairs + (size_t)(j & 1) * kSetCtas * kSlotWords;
+        // partial rows of split tiles: [set j & 1][CTA][matrix][row][column]
+        float* set_parts = sp.ws.parts + (size_t)(j & 1) * kSetCtas * kSlotWords;
         const size_t row_off = (size_t)rw * kTileN + 4 * lane;
 
         if (!whole && !finish) {
-          // ---- contributor: row r of its partial tile as {value, tag} pairs; nothing else to do.
-          //      (A run that does not begin its tile meets it in its first segment, so one slot
-          //      per CTA is enough.) ----
+          // ---- contributor: row r of its partial tile; nothing else to do.  (A run that does not
+          //      begin its tile meets it in its first segment, so one slot per CTA is enough.) ----
           for (int mt = 0; mt < nmat; ++mt) {
             const float* f = mt ? f1 : f0;
-            uint64_t* dst = set_pairs + (size_t)cta * kSlotWords + (size_t)mt * MP * kTileN + row_off;
-            st_pairs(dst, f[0], f[1], tag);
-            st_pairs(dst + 2, f[2], f[3], tag);
+            st_part(set_parts + (size_t)cta * kSlotWords + (size_t)mt * MP * kTileN + row_off, f[0], f[1], f[2], f[3]);
           }
           if (pos - nch == start) QL_STAMP(6);
           if (pos == end) QL_STAMP(14);
@@ -870,32 +873,31 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
         }
         if (!whole && !(sp.ablate & 8)) {
           // ---- owner of a split tile: its own partial stays in registers; the others' rows are
-          //      polled until every pair carries this operation's tag and added in CTA order ----
+          //      polled until no word is empty any more, added in CTA order, and their slots emptied ----
           const uint32_t last = h.last;                  // (a split tile that a piece begins is the piece's last tile)
           if (pos == end) QL_STAMP(10);
           // items = (contributor, matrix) in CTA order, the two matrices of a dual operation side by
-          // side: four items are in flight together (one round of loads covers two contributors of a
-          // gate/up pair or four of a plain linear)
+          // side: in chains eight items are in flight together (one round of loads covers every tile of
+          // the verify step: at most 7 contributors of a plain linear, 2 or 3 of a gate/up pair)
+          constexpr int GB = PAIRED ? 8 : 4;             // (the variants for streams have 80 registers and few contributors)
           const uint32_t items = (last - cta) * (uint32_t)nmat;
-          for (uint32_t k0 = 0; k0 < items; k0 += 4) {
-            uint64_t u[4][4];
+          for (uint32_t k0 = 0; k0 < items; k0 += GB) {
+            uint32_t u[GB][4];
             uint64_t t0 = 0;
             uint32_t spins = 0;
             for (;;) {
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
+              for (int q = 0; q < GB; ++q) {
                 const uint32_t k = min(k0 + q, items - 1);
                 const uint32_t i = cta + 1 + (dual ? (k >> 1) : k);
                 const uint32_t mt = dual ? (k & 1u) : 0u;
-                const uint64_t* src = set_pairs + (size_t)i * kSlotWords + (size_t)mt * MP * kTileN + row_off;
-                ld_pairs(src, u[q][0], u[q][1]);
-                ld_pairs(src + 2, u[q][2], u[q][3]);
+                ld_part(set_parts + (size_t)i * kSlotWords + (size_t)mt * MP * kTileN + row_off, u[q]);
               }
               bool ok = true;
 #pragma unroll
-              for (int q = 0; q < 4; ++q)
+              for (int q = 0; q < GB; ++q)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) ok = ok && ((uint32_t)(u[q][e] >> 32) == tag);
+                for (int e = 0; e < 4; ++e) ok = ok && (u[q][e] != kPartEmpty);
               if (ok) break;
               if (spins == 0) {
                 if (*wc.s_abort) break;
@@ -907,12 +909,16 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
               }
             }
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
+            for (int q = 0; q < GB; ++q) {
               if (k0 + q >= items) continue;
-              const float a0 = __uint_as_float((uint32_t)u[q][0]), a1 = __uint_as_float((uint32_t)u[q][1]);
-              const float a2 = __uint_as_float((uint32_t)u[q][2]), a3 = __uint_as_float((uint32_t)u[q][3]);
-              if (dual && (q & 1)) { f1[0] += a0; f1[1] += a1; f1[2] += a2; f1[3] += a3; }   // (k0 is a multiple of 4: item parity = q parity)
+              const float a0 = __uint_as_float(u[q][0]), a1 = __uint_as_float(u[q][1]);
+              const float a2 = __uint_as_float(u[q][2]), a3 = __uint_as_float(u[q][3]);
+              if (dual && (q & 1)) { f1[0] += a0; f1[1] += a1; f1[2] += a2; f1[3] += a3; }   // (k0 is even: item parity = q parity)
               else { f0[0] += a0; f0[1] += a1; f0[2] += a2; f0[3] += a3; }
+              const uint32_t k = k0 + q;
+              const uint32_t i = cta + 1 + (dual ? (k >> 1) : k);
+              const uint32_t mt = dual ? (k & 1u) : 0u;
+              clear_part(set_parts + (size_t)i * kSlotWords + (size_t)mt * MP * kTileN + row_off);
             }
           }
           __syncwarp();

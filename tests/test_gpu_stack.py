@@ -146,6 +146,33 @@ def test_full_size_layer_under_every_split(ql, g):
         ql.ql_debug_set_owner_extra(-1)
 
 
+def test_nan_rows_propagate_through_split_tiles(ql):
+    """Partial rows of split tiles signal themselves by not being the 'empty' bit pattern (an
+    all-ones NaN).  Rows of X that are NaN - the canonical one and the all-ones one - must come out
+    as NaN rows without stalling the exchange; the other rows still match the oracle."""
+    M, g = 16, 128
+    K, N = qsynth.LAYER_SHAPES["o"]
+    lin = qsynth.make_linear([77, 3], M, K, N, g)
+    x = lin["x"].copy()
+    x[3, :] = 0x7FC0
+    x[9, :] = 0xFFFF
+    y = torch.zeros((M, N), dtype=torch.int16, device="cuda")
+    ops = ql.make_ops([dict(kind=ql.QL_OP_LINEAR, M=M, K=K, N=N, g=g, ld_in=K, ld_out=N, packed=pack_on_device(ql, lin),
+                            in0=dev_u16(x), out=y)])
+    ws = ql.new_workspace(M, N)
+    assert ql.ql_plan_chain_split(N // 128, K // g, 148, 0)["aligned"]
+    for _ in range(2):
+        ql.qlinear_stack_w4a16(ops, ws)
+        torch.cuda.synchronize()
+        assert ql.ql_device_status(ws) == ql.QL_OK
+        got = host_u16(y)
+        for r in (3, 9):
+            assert np.all((got[r] & 0x7F80) == 0x7F80) and np.all((got[r] & 0x007F) != 0), f"row {r} is not NaN throughout"
+        keep = [r for r in range(M) if r not in (3, 9)]
+        want = orc.qlinear_f64(lin["x"], lin["wq"], lin["scale"], lin["zero"], g)
+        check_against_oracle(got[keep], want[keep], "rows beside the NaN rows")
+
+
 def test_drafter_layers_symmetric_full_size(ql):
     """The second workload: drafter layers (group-wise symmetric INT4, groups of 128, M = 16; paper
     Sections 3.2 and 3.3) through the same launcher, zero == NULL at the boundary.  Two of the five

@@ -177,7 +177,7 @@ def test_chain_split_aligned_where_tiles_can_have_thread_blocks_of_their_own(ql)
                     nc = min(ncta, total)
                     assert [r["lo"] for r in rs[:nc]] == [(i * total) // nc for i in range(nc)]
                     continue
-                e = 1 if extra == -1 else extra
+                e = 0 if extra == -1 else extra
                 for T in range(nt):
                     ctas = [i for i, r in enumerate(rs) if r["lo"] // gn == T]
                     assert ctas == list(range(ctas[0], ctas[-1] + 1)) and len(ctas) >= 2
