@@ -23,7 +23,7 @@ cudaError_t launch_stack_tc5(const StackParams& sp, int g, size_t smem, cudaStre
 cudaError_t launch_unit_rms(const uint16_t*, const uint16_t*, uint16_t*, int, int, int, int, bool, cudaStream_t);
 
 static std::atomic<uint64_t> g_launches{0};
-static std::atomic<uint32_t> g_epoch{0};                  // stack-kernel launches: tags of split-K partial tiles
+static std::atomic<uint32_t> g_epoch{0};                  // stack-kernel launches so far
 static std::atomic<uint64_t> g_wait_ns{kWaitBudgetNs};    // budget of the stack kernel's bounded waits
 // Bumped whenever operation descriptors are staged into any workspace, a workspace is re-initialised or a
 // debug hook changes: a remembered plan is valid only while nothing of that happened since it was staged.

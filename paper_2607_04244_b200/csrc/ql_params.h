@@ -78,7 +78,7 @@ struct StackParams {
                            // linears): the X slots are a ring of P chunks filled by a loader warp, chunk by chunk
   int one_stream;          // the operations are independent plain linears laid end to end (selects the kernel variant)
   int ablate;              // timing experiments only (see the stack kernel); 0 in production
-  uint32_t epoch;          // launch number: partial tiles in the workspace carry (epoch, operation) tags
+  uint32_t epoch;          // launch number (kept for diagnostics; nothing in the kernel depends on it)
   uint64_t wait_ns;        // budget of every bounded wait
   uint64_t* timeline;      // builds with -DQL_TIMELINE only: [ncta][n_ops][8] globaltimer stamps, else nullptr
   Workspace ws;

@@ -25,13 +25,13 @@
 //   * a group owns three half-chunk A buffers in tensor memory and unpacks the first one and a
 //     half chunks of operation j+1 BEFORE its X exists (the A operand depends on weights only);
 //     the issuers hold the MMAs back until X has been published;
-//   * waiting is done with relaxed loads (no fence per poll); the one acquire fence follows the
-//     successful poll;
+//   * waiting is done with relaxed loads (no fence per poll); one acquire load per counter follows
+//     the successful poll;
 //   * the end of a tile is handled row by row: after one exchange through shared memory warp r owns
 //     row r, and from there on the 16 warps never meet again - a contributor's warp stores its row
-//     of the partial tile, fences and raises the row's flag (tagged with launch and operation
-//     number, so flags are never reset); the owner's warp r polls the contributors' row flags, adds
-//     their rows in CTA order (deterministic, no floating-point atomics), stores the bf16 row and the
+//     of the partial tile into its slot, whose words are an "empty" bit pattern until a value lands;
+//     the owner's warp r polls the contributors' slots until no word is empty, adds the rows in CTA
+//     order, puts the empty pattern back (deterministic, no floating-point atomics), stores the bf16 row and the
 //     row's sum of squares and publishes the row to a per-row counter of the operation;
 //   * the glue between linears is folded in: a finished tile also leaves the row sums of squares
 //     of what the next operation normalises, and that operation builds its X operand as
@@ -712,7 +712,6 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
       const bool dual = (h.flags & kOpDual) != 0;
       const uint32_t Gn = (uint32_t)h.n_groups;
       const uint32_t my_chunks = end - start;
-      const uint32_t tag = (sp.epoch << 9) | (uint32_t)(j + 1);
       const uint32_t n_sub_total = my_chunks * (dual ? 2u : 1u);
       QL_STAMP(0);
 
@@ -812,9 +811,11 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
         if (!(sp.ablate & 1)) {
           if (n_pend == 2) drain(kloc - 2, s_p2);
           if (n_pend >= 1) drain(kloc - 1, s_p1);
-          // nobody waits for this tile: the group's first chunk of the NEXT segment is unpacked
-          // before this segment's tile end, so that its MMAs run while the rows are finished
-          if ((h.flags & kOpLazy) && e_own < n_sub_total && !pre_done) {
+          // a segment that is not the piece's last: the group's first chunk of the NEXT segment is
+          // unpacked before this segment's tile end, so that its MMAs run while the rows are finished
+          // (the tile of a segment in the middle of a piece is a whole one, or one whose owner gathers
+          // the partial rows at the end of ITS piece: nobody waits for it yet)
+          if (e_own < n_sub_total && !pre_done) {
             pre_sc = unpack_subchunk(s_own, ph_own);
             pre_done = true;
           }
