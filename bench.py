@@ -35,9 +35,9 @@ import qsynth  # noqa: E402
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from an ncu capture of a 3-layer launch of the stack kernel:
-# dram read + write = 160.95 MB for 162.32 MB of algorithmic bytes.  Traffic grows in proportion to the
+# dram read + write = 161.91 MB for 162.32 MB of algorithmic bytes.  Traffic grows in proportion to the
 # layers streamed (every packed byte crosses HBM once), so a full launch is scaled by this ratio.
-NCU_TRAFFIC_RATIO = 161.42 / 162.32
+NCU_TRAFFIC_RATIO = 161.91 / 162.32
 
 
 # ------------------------------------------------------------------------------------------------
