@@ -74,10 +74,12 @@ size_t ql_packed_bytes(int K, int N, int g);
  * word).  Returns 0 for unsupported arguments.  Needs no device. */
 size_t ql_workspace_bytes(int M_max, int N_max);
 
-/* Zeroes a workspace (asynchronously, on `stream`): its control words, and the partial-tile slots,
- * whose entries carry a tag that must not look valid by accident.  Call once after allocating the
- * workspace, and again after a call reported QL_ERR_DEVICE_TIMEOUT.  The kernels leave the control
- * words zeroed when they finish, so no further initialisation is needed between calls.  One
+/* Initialises a workspace (asynchronously, on `stream`): zero everywhere, except for the region
+ * through which thread blocks of qlinear_stack_w4a16 hand partial rows to one another, which is
+ * filled with the bit pattern that means "nothing waiting" (all ones).  Call once after allocating
+ * the workspace, after the memory was used for anything else (the attention call included), and
+ * again after a call reported QL_ERR_DEVICE_TIMEOUT.  The kernels leave the control words zeroed
+ * and that region empty when they finish, so no further initialisation is needed between calls.  One
  * workspace serves one stream at a time: calls that may overlap on the GPU need separate
  * workspaces. */
 int ql_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
