@@ -40,7 +40,7 @@ def test_two_rank_aggregation_on_gloo():
         assert val == pytest.approx(2 * 1.0 / 3.5e-3)                    # 2 GB over 3.5 ms, in GB/s
 
 
-def test_byte_accounting_matches_the_survey_figures():
+def test_byte_accounting_of_the_algorithmic_bytes():
     sys.path.insert(0, ROOT)
     import bench
     assert bench.linear_bytes(16, 2560, 9728, 128) == 13_331_456
