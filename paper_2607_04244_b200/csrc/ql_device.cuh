@@ -16,9 +16,9 @@ __host__ __device__ constexpr uint32_t align128(uint32_t x) { return (x + 127u) 
 // ---- workspace layout -----------------------------------------------------------------------
 // [0, 256)        control header: word 0 status, word 1 finished-tile counter (arg-max),
 //                 word 2 finished-CTA counter of the stack kernel
-// then            per-tile arrival counters (split-K) of the single-linear kernels [kMaxTiles], followed by the
-//                 partial-row flags of the stack kernel [2][160][16] (tagged with launch and operation, never
-//                 reset, hence in words of their own)              [kFlagWords in all]
+// then            per-tile arrival counters (split-K) of the single-linear kernels [kMaxTiles], a reserved
+//                 block [2][160][16], the stack kernel's per-row arg-max counters and its verification-tail
+//                 counter on lines of their own                    [kFlagWords in all]
 // then            per-operation, per-row finished-tile counters of the stack kernel, one 128-byte line each
 //                                                                [kMaxOps][16][32]
 // -- everything above is zero between calls (ql_workspace_init zeroes it once, kernels restore it) --
@@ -26,12 +26,12 @@ __host__ __device__ constexpr uint32_t align128(uint32_t x) { return (x + 127u) 
 // then            partial tiles of the stack kernel (self-signalling values)   [kWsPairBytes]
 // then            row sums of squares per tile, two buffers      [2][tiles][16] fp32
 // then            fp32 product silu(gate)*up of a dual operation, dense [16][N]   [16][tiles*128]
-// then            arg-max candidates                             [tiles][m_pad] (value, index)
+// then            arg-max candidates                             [m_pad][tiles] (value, index)
 // then            split-K partial tiles  [kMaxCtas][2 segments][2 matrices][m_pad*128] fp32
 constexpr int kMaxCtas = 320;                     // up to two CTAs per SM
 constexpr int kMaxTiles = 4096;                   // N <= 128 * 4096
-constexpr int kStackFlagWords = 2 * 160 * 16;      // partial-row flags of the stack kernel: [2 sets][160 CTAs][16 rows]
-constexpr int kFlagWords = kMaxTiles + kStackFlagWords + 1024;   // tile counters [kMaxTiles], then the stack kernel's flags (tagged, never reset: they must not alias the counters), then its 16 per-row arg-max counters and its verification-tail counter on lines of their own
+constexpr int kStackFlagWords = 2 * 160 * 16;      // reserved (row flags of an earlier exchange scheme; the words stay zero)
+constexpr int kFlagWords = kMaxTiles + kStackFlagWords + 1024;   // tile counters [kMaxTiles], the reserved block, then the stack kernel's 16 per-row arg-max counters and its verification-tail counter on lines of their own
 constexpr int kMaxOps = 256;                      // fused operations per stack-kernel launch
 constexpr int kOpDoneStride = 32;                 // ints between the counters of two rows (one line each: they are polled)
 constexpr int kOpDescBytes = 160;

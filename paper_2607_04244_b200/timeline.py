@@ -149,7 +149,7 @@ def main():
             "last segment: accumulator exchange (mean)": mean(e[:, 9] - e[:, 8]),
             "owners of split tiles: exchange -> polling starts (mean)": mean(e[:, 10] - e[:, 9]),
             "owners of split tiles: exchange -> polling starts (max)": vmax(e[:, 10] - e[:, 9]),
-            "owners: poll and add the contributors' tagged rows (mean)": mean(e[:, 11] - e[:, 10]),
+            "owners: poll and add the contributors' rows (mean)": mean(e[:, 11] - e[:, 10]),
             "finishers: epilogue until stores issued (mean)": mean(e[:, 12] - e[:, 11]),
             "finishers: fence + publish (mean)": mean(e[:, 14] - e[:, 12]),
             "contributors: exchange -> partial sent (mean)": mean(np.where(np.isnan(e[:, 11]), e[:, 14] - e[:, 9], np.nan)),
