@@ -512,10 +512,13 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
       // an operation waits for the one before it (it consumes its output), or only for the one two
       // back (independent operations: the partial-tile slots and flags alternate between two sets)
       const int dep = (h.flags & kOpWait) ? j - 1 : -1;
+      // (read before the wait: after it, every load is on the path to the next operation's X)
+      const int prologue = __ldg(&ops[j].prologue);
+      const int src_tiles = __ldg(&ops[j].src_tiles);
       if (dep >= 0) {
         // every tile is published row by row; lane r polls the counter of row r (one line per counter)
         if (lane < 16) {
-          const int need = __ldg(&ops[dep].n_tiles);
+          const int need = load_head(s_heads, dep).n_tiles;
           wait_global<true>(&sp.ws.op_done[((size_t)dep * 16 + lane) * kOpDoneStride], need, wc, 7);
         }
         // acquire: everything the finishers published.  One acquire load of the complete counter per
@@ -528,13 +531,11 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
         __threadfence_block();
         *s_dep = j + 1;
       }
-      const int prologue = __ldg(&ops[j].prologue);
       uint32_t start, end;
       start = h.start; end = h.end;
       if (prologue != 0 && start < end) {
         // 1/rms of every row from the per-tile sums of squares the producer operation left
         // (fixed order: tiles of one parity ascending, then even + odd)
-        const int src_tiles = __ldg(&ops[j].src_tiles);
         const float* ssq = sp.ws.ssq + (size_t)((j - 1) & 1) * sp.ws.n_tiles * 16;
         const int row = lane & 15, half = lane >> 4;
         float sum = 0.f;
