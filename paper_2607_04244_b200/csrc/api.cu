@@ -539,8 +539,8 @@ int ql_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
   // everything, not only the control words; the stack kernel's partial-tile region holds "nothing waiting" (all ones)
   if (cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) return QL_ERR_CUDA;
   const size_t parts_at = kWsControlBytes + kWsDescBytes;
-  if (workspace_bytes >= parts_at + kWsPairBytes &&
-      cudaMemsetAsync(static_cast<char*>(workspace) + parts_at, 0xFF, kWsPairBytes, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+  if (workspace_bytes >= parts_at + kWsPartBytes &&
+      cudaMemsetAsync(static_cast<char*>(workspace) + parts_at, 0xFF, kWsPartBytes, static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return QL_ERR_CUDA;
   return QL_OK;
 }

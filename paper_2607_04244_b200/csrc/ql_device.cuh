@@ -23,7 +23,7 @@ __host__ __device__ constexpr uint32_t align128(uint32_t x) { return (x + 127u) 
 //                                                                [kMaxOps][16][32]
 // -- everything above is zero between calls (ql_workspace_init zeroes it once, kernels restore it) --
 // then            operation descriptors of the stack kernel      [kMaxOps * kOpDescBytes]
-// then            partial tiles of the stack kernel (self-signalling values)   [kWsPairBytes]
+// then            partial tiles of the stack kernel (self-signalling values)   [kWsPartBytes]
 // then            row sums of squares per tile, two buffers      [2][tiles][16] fp32
 // then            fp32 product silu(gate)*up of a dual operation, dense [16][N]   [16][tiles*128]
 // then            arg-max candidates                             [m_pad][tiles] (value, index)
@@ -43,7 +43,7 @@ constexpr size_t kWsDescBytes = (size_t)kMaxOps * kOpDescBytes;
 // it back) or a value a contributor stored: the value is its own signal, no flag and no fence travel
 // with it.  The region is written by that kernel only and sits at a fixed offset.
 constexpr uint32_t kPartEmpty = 0xFFFFFFFFu;         // a NaN no arithmetic produces (stores replace it by the canonical NaN)
-constexpr size_t kWsPairBytes = (size_t)kMaxCtas * 2 * 16 * 128 * 4;
+constexpr size_t kWsPartBytes = (size_t)kMaxCtas * 2 * 16 * 128 * 4;
 
 struct Workspace {
   int* status;
@@ -67,7 +67,7 @@ __host__ __device__ inline size_t ws_cand_bytes(int n_tiles, int m_pad) { return
 __host__ __device__ inline size_t ws_slot_floats(int m_pad) { return (size_t)2 * m_pad * kTileN; }   // two matrices
 __host__ __device__ inline size_t ws_act_bytes(int n_tiles) { return (size_t)16 * n_tiles * kTileN * 4; }
 __host__ __device__ inline size_t ws_total_bytes(int n_tiles, int m_pad) {
-  return kWsControlBytes + kWsDescBytes + kWsPairBytes + ws_ssq_bytes(n_tiles) + ws_act_bytes(n_tiles) + ws_cand_bytes(n_tiles, m_pad) +
+  return kWsControlBytes + kWsDescBytes + kWsPartBytes + ws_ssq_bytes(n_tiles) + ws_act_bytes(n_tiles) + ws_cand_bytes(n_tiles, m_pad) +
          (size_t)kMaxCtas * 2 * ws_slot_floats(m_pad) * 4;
 }
 // Carves the regions for a tile capacity and row padding.  Within one workspace every call must
@@ -83,7 +83,7 @@ __host__ __device__ inline Workspace ws_carve(void* base, int n_tiles, int m_pad
   w.op_done = w.tile_cnt + kFlagWords;
   w.desc = (uint8_t*)(p + kWsControlBytes);
   w.parts = (float*)(p + kWsControlBytes + kWsDescBytes);
-  p += kWsControlBytes + kWsDescBytes + kWsPairBytes;
+  p += kWsControlBytes + kWsDescBytes + kWsPartBytes;
   w.ssq = (float*)p;
   p += ws_ssq_bytes(n_tiles);
   w.act = (float*)p;
