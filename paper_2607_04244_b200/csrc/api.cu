@@ -96,13 +96,14 @@ static int prepare_linear(LinearParams& p, const void* packed, const uint16_t* X
 }
 
 // Path choice for a linear launched on its own (measured with `bench.py --paths`, 24 cold weight
-// sets, one launch per linear): up to 16 rows the warp-level mma.sync kernel is 1-6 us faster than
-// the tcgen05 kernel (18.9 vs 20.2-22.1 us at 2560x9728: both are latency-bound, and the tcgen05
-// kernel pays for the tensor-memory allocation and a second barrier hop per chunk); at 32 rows they
-// are equal, at 64 rows tcgen05 wins where its X operand fits in shared memory.  (The persistent
-// stack and batch kernels, which the stack launcher uses for M <= 16, are tcgen05 kernels.)
+// sets, one launch per linear): up to 32 rows the warp-level mma.sync kernel is faster than the
+// tcgen05 kernel (11.5-16 us against 17-26 us up to 16 rows, 15.8-21.6 against 18.8-23 at 32 rows:
+// both are latency-bound, the tcgen05 kernel pays for the tensor-memory allocation and a second
+// barrier hop per chunk, and the mma.sync kernel's launches overlap their set-up with the
+// predecessor's tail); at 64 rows tcgen05 wins where its X operand fits in shared memory.  (The
+// persistent stack kernel, which the stack launcher uses for M <= 16, is a tcgen05 kernel.)
 static int select_path(const LinearParams& p, int sms) {
-  if (p.M <= 16) return QL_PATH_MMA;
+  if (p.M <= 32) return QL_PATH_MMA;
   return tc5_supported(p, sms) ? QL_PATH_TC5 : QL_PATH_MMA;
 }
 

@@ -133,10 +133,17 @@ __global__ void __launch_bounds__(mma_kgroups(MT) * 128 + 32, 1) qlinear_mma_ker
   }
   __syncthreads();
 
+  // Programmatic dependent launch: the next kernel of the stream may be scheduled as soon as every CTA of
+  // this one has got here (its CTAs start where SMs become free, and their set-up overlaps this
+  // kernel's tail).  Nothing a kernel does before its own griddepcontrol.wait may depend on the
+  // kernels before it: here that is the barrier set-up only.
+  grid_dep_launch();
+
   if (warp == KG * 4) {
     // ------------------------------------------------------------------ producer
     uint32_t it = 0;
     if (lane == 0) {
+      grid_dep_wait();                                   // the packed weights may be the previous kernel's output
       const uint64_t pol = policy_evict_first();
       const uint32_t cb = chunk_bytes(G);
       const uint8_t* src = p.packed + (size_t)start * cb;
@@ -165,6 +172,8 @@ __global__ void __launch_bounds__(mma_kgroups(MT) * 128 + 32, 1) qlinear_mma_ker
 
   // -------------------------------------------------------------------- consumers
   const int kg = warp >> 2, wn = warp & 3, g8 = lane >> 2, t = lane & 3;
+  // X, the workspace and Y belong to the kernels before this one until they have completed
+  grid_dep_wait();
   const size_t slot_f4 = ws_slot_floats(p.m_pad) / 4;
   const uint32_t g_first = start % Gn;
   // X staging: slot k of xbuf receives the X columns of the group of the CTA's chunk number
@@ -397,8 +406,17 @@ static cudaError_t launch_one(const LinearParams& p, size_t smem, cudaStream_t s
     if (e != cudaSuccess) return e;
     attr_set[dev] = true;
   }
-  qlinear_mma_kernel<MT, G><<<p.ncta, mma_kgroups(MT) * 128 + 32, smem, stream>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.ncta);
+  cfg.blockDim = dim3(mma_kgroups(MT) * 128 + 32);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see grid_dep_launch / grid_dep_wait in the kernel
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, qlinear_mma_kernel<MT, G>, p);
 }
 
 // Fills the path-specific fields of `p` (ring depth, X slots, resident or phased X); returns the

@@ -41,10 +41,12 @@ PATHS = [pytest.param(2, id="mma"), pytest.param(3, id="tcgen05")]
 
 def _skip_unless_supported(ql, path, M, K, N, g):
     """The tcgen05 kernel needs the X columns a CTA touches to fit in shared memory.  Up to 16 rows
-    they always do for these shapes; above, ql_select_path answers tcgen05 exactly when they fit."""
+    they always do for these shapes; above, the plan for the forced path says whether they fit."""
     if path != ql.QL_PATH_TC5:
         return
-    if M > 16 and ql.ql_select_path(M, K, N, g) != ql.QL_PATH_TC5:
+    try:
+        ql.ql_linear_plan(M, K, N, g, ql.QL_PATH_TC5)
+    except ql.QlError:
         pytest.skip("X does not fit in shared memory for the tcgen05 path at this shape")
 
 
