@@ -78,7 +78,9 @@ size_t ql_workspace_bytes(int M_max, int N_max);
  * through which thread blocks of qlinear_stack_w4a16 hand partial rows to one another, which is
  * filled with the bit pattern that means "nothing waiting" (all ones).  Call once after allocating
  * the workspace, after the memory was used for anything else (the attention call included), and
- * again after a call reported QL_ERR_DEVICE_TIMEOUT.  The kernels leave the control words zeroed
+ * again after a call reported QL_ERR_DEVICE_TIMEOUT (until then the status word stays set, and
+ * qlinear_stack_w4a16 launches on that workspace run through without waiting for anything: their
+ * results are not valid, and ql_device_status keeps saying why).  The kernels leave the control words zeroed
  * and that region empty when they finish, so no further initialisation is needed between calls.  One
  * workspace serves one stream at a time: calls that may overlap on the GPU need separate
  * workspaces. */

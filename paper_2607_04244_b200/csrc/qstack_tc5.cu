@@ -423,7 +423,10 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
       mbar_init(&xr_full[i], 32);                        // the loader's 32 lanes, each when its copies have landed
       mbar_init(&xr_empty[i], 1);
     }
-    *s_abort = 0;
+    // a status word that is still set means an earlier launch gave up on this workspace and nobody has
+    // initialised it again: its counters and partial-tile slots cannot be trusted, so this launch
+    // does not wait for anything either (it runs through, and the status keeps saying why)
+    *s_abort = ld_relaxed(sp.ws.status) != 0 ? 1 : 0;
     *s_dep = 0;
     *s_invrdy = 0;
     *s_descrdy = 0;

@@ -40,6 +40,14 @@ def test_wait_runs_out_reports_and_recovers(ql):
     raw = ql.ql_device_status_raw(ws)
     site = (raw >> 8) & 0xFF
     assert site == 7, f"expected the watcher's poll of the predecessor (site 7), got site {site}"
+    # a launch on the workspace as the timeout left it (hook off, full 2 s budget) must not wait for
+    # anything: it runs through at once and the status keeps reporting the timeout
+    import time
+    t0 = time.perf_counter()
+    ql.qlinear_stack_w4a16(ops, ws)
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 1.0
+    assert ql.ql_device_status(ws) == ql.QL_ERR_DEVICE_TIMEOUT
     # recovery: re-initialise the workspace, run the same list for real
     ql.ql_workspace_init(ws)
     y1.zero_(); y2.zero_()
