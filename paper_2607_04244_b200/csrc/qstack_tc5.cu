@@ -814,15 +814,17 @@ __global__ void __launch_bounds__(st_threads(RING, PAIRED), 1) qstack_tc5_kernel
         }
         if (!(sp.ablate & 1)) {
           if (n_pend == 2) drain(kloc - 2, s_p2);
-          if (n_pend >= 1) drain(kloc - 1, s_p1);
           // a segment that is not the piece's last: the group's first chunk of the NEXT segment is
           // unpacked before this segment's tile end, so that its MMAs run while the rows are finished
           // (the tile of a segment in the middle of a piece is a whole one, or one whose owner gathers
-          // the partial rows at the end of ITS piece: nobody waits for it yet)
+          // the partial rows at the end of ITS piece: nobody waits for it yet) - and before the last
+          // chunk of this segment is read back: its MMAs were handed over a moment ago, and the
+          // accumulator buffer the new chunk will use is the one just drained
           if (e_own < n_sub_total && !pre_done) {
             pre_sc = unpack_subchunk(s_own, ph_own);
             pre_done = true;
           }
+          if (n_pend >= 1) drain(kloc - 1, s_p1);
         }
         tc_fence_before_sync();
 #ifdef QL_TIMELINE
