@@ -310,6 +310,8 @@ static int run_stack(const ql_op* ops, int n_ops, void* workspace, size_t worksp
           chain_split(m, ncta);
           if (j > 0) m.flags |= kOpWait;
         }
+        mega.back().flags |= kOpLazy;   // nothing in the launch waits for the last operation: its rows need not be published
+
       }
       const int hook = g_no_release_op.load(std::memory_order_relaxed);
       if (hook >= 0 && hook < (int)mega.size()) mega[hook].flags |= kOpNoRelease;

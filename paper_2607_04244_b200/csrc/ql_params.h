@@ -36,8 +36,8 @@ struct LinearParams {
 // The first 32 bytes hold what every role reads at every operation.
 constexpr int kOpDual = 1;        // two matrices (packed0, packed1) share X
 constexpr int kOpWait = 2;        // X may be read only after operation j-1 has finished every tile
-constexpr int kOpLazy = 16;       // nothing in the launch waits for this operation's tiles: they need not be published, and the
-                                  // next tile segment may be started before the current one is finished
+constexpr int kOpLazy = 16;       // nothing in the launch waits for this operation's tiles (independent linears of one stream, the
+                                  // last operation of a chain): they need not be published
 constexpr int kOpNoRelease = 4;   // test hook: finished tiles are not published (the next operation's wait runs out)
 struct MegaOp {
   uint32_t nc, cq, cr;     // CTA i owns run positions [i*cq + i*cr/nc, (i+1)*cq + (i+1)*cr/nc), i < nc; or, with
